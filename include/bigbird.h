@@ -1,0 +1,151 @@
+/*
+ * bigbird.h -- C ABI of the BigBird block-sparse attention forward library for NVIDIA B200 (sm_100a).
+ *
+ * The operation is the generalised attention of arXiv 2007.14062, Sec. 2, Eq. (AT), restricted to its
+ * per-head softmax core:
+ *
+ *     out[i] = sum_{k in N(i)} softmax_k( scale * q_i . k_k ) v_k ,    lse[i] = ln sum_{k in N(i)} exp(scale * q_i . k_k)
+ *
+ * where the out-neighbour sets N(i) are those of the block-sparse BigBird graph of App. D: with the
+ * sequence cut into blocks of b tokens, query block j attends to the w key blocks of its sliding window
+ * (j-(w-1)/2 .. j+(w-1)/2), to the g global blocks and to r random key blocks; global query blocks attend
+ * to every block (Sec. 2: A(i,:) = A(:,i) = 1 for i in G).  ITC makes existing blocks global, ETC puts the
+ * global tokens in front of the sequence (matrix B of Sec. 2).
+ *
+ * Conventions
+ *   - every function returns BIGBIRD_OK (0) or a negative error code; nothing throws, aborts or traps;
+ *   - "host" / "device" in a comment says where the pointer must live;
+ *   - the caller owns every buffer it passes; the library owns layout handles until they are destroyed;
+ *   - one GPU per call: the device that is current on the calling thread.
+ */
+#ifndef BIGBIRD_H_
+#define BIGBIRD_H_
+
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define BIGBIRD_API __attribute__((visibility("default")))
+#else
+#define BIGBIRD_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    BIGBIRD_OK = 0,
+    BIGBIRD_EINVAL = -1,        /* null pointer, N % b != 0, even w, g > N/b, layout built for another N/b/H ... */
+    BIGBIRD_EUNSUPPORTED = -2,  /* shape or dtype outside what the kernels implement */
+    BIGBIRD_ECUDA = -3,         /* a CUDA call failed; see bigbird_last_cuda_error() */
+    BIGBIRD_ETIMEOUT = -4,      /* a bounded wait inside a kernel expired (reported by bigbird_last_status) */
+    BIGBIRD_ENOMEM = -5
+};
+
+enum { BIGBIRD_ITC = 0, BIGBIRD_ETC = 1 };
+enum { BIGBIRD_FP32 = 0, BIGBIRD_BF16 = 1 };
+
+typedef struct bigbird_layout bigbird_layout;   /* opaque */
+
+/*
+ * bigbird_build_layout -- the attention graph of App. D as per-(head, query block) key-block lists.
+ *
+ *   N     total tokens per sequence (ETC: including the prepended global tokens); N % b == 0
+ *   b     block size in tokens
+ *   w     sliding-window width in blocks, odd: query block j sees key blocks j-(w-1)/2 .. j+(w-1)/2,
+ *         clipped at the ends of the sequence (App. D item 2)
+ *   g     number of global blocks (Sec. 2; App. D item 3).  mode BIGBIRD_ITC: the first ceil(g/2) and the last
+ *         floor(g/2) blocks; mode BIGBIRD_ETC: the first g blocks
+ *   r     random key blocks per (head, non-global query block) (App. D item 1), drawn without replacement
+ *         from the ascending list of blocks that are neither in the query block's window nor global (all of
+ *         them if fewer than r).  The same for every batch element; not symmetrised (the graph is directed).
+ *   seed  selects the random blocks.  The paper fixes no generator; this library's is: a SplitMix64 stream
+ *         with initial state (seed << 40) ^ (h << 20) ^ j for head h and query block j (h, j < 2^20), the
+ *         bounded draw floor(z * m / 2^64), and a partial Fisher-Yates shuffle of the candidate list
+ *         (for t < r: swap entries t and t + draw(m - t)); the first r entries are taken.
+ *   H     number of heads
+ *
+ * Row (h, j) of the result lists its key blocks in ascending order without duplicates; a global query
+ * block lists all N/b blocks.  The handle also carries the device-side schedule derived from the lists;
+ * device memory for it is allocated on the first bigbird_attn_fwd that uses the handle.
+ * Host-only; thread-safe for distinct handles.  Errors: BIGBIRD_EINVAL, BIGBIRD_ENOMEM.
+ */
+BIGBIRD_API int bigbird_build_layout(int64_t N, int b, int w, int g, int r, uint64_t seed, int H, int mode,
+                         bigbird_layout** out_layout);
+
+/* Number of listed (query block, key block) pairs, summed over heads. */
+BIGBIRD_API int bigbird_layout_nnz(const bigbird_layout* layout, int64_t* nnz);
+
+/* Copies the lists out as CSR over rows h * (N/b) + j.  row_ptr: host int32[H * N/b + 1];
+ * col_idx: host int32[nnz].  Both caller-owned. */
+BIGBIRD_API int bigbird_layout_export(const bigbird_layout* layout, int32_t* row_ptr, int32_t* col_idx);
+
+/*
+ * Introspection of the tile schedule derived from the lists (used by the tests; not needed to run attention).
+ * The tensor-core kernel stacks two query blocks into one 2b-row tile and walks a list of steps: a full step
+ * is one key block attended by both halves of the tile, a split step pairs a key block attended only by the
+ * upper half with one attended only by the lower half.
+ *   sizes   host int32[4]: items per head, leading "heavy" (global-tile) items per head, total steps, heads
+ *   items   host int32[H * items_per_head * 8] or NULL: per item (qa, qb, step_begin, step_count, part, nparts, tile, 0),
+ *           step_begin relative to the head's first step
+ *   step_base host int32[H] or NULL: first step of each head
+ *   steps   host int32[total_steps * 2] or NULL: (c0, c1); c1 == -2 marks a full step, -1 marks "no block"
+ */
+BIGBIRD_API int bigbird_layout_schedule(const bigbird_layout* layout, int32_t* sizes, int32_t* items, int32_t* step_base,
+                            int32_t* steps);
+
+/* Frees the handle and the device memory it holds.  No kernel using it may still be running. */
+BIGBIRD_API int bigbird_layout_destroy(bigbird_layout* layout);
+
+/*
+ * bigbird_attn_fwd -- Eq. (AT) over the graph held by `layout`, for every batch element and head.
+ *
+ *   q, k, v   device, [B, H, N, D] contiguous, fp32 or bf16 according to `dtype`; 16-byte aligned
+ *   layout    from bigbird_build_layout with the same N, b, H
+ *   key_padding_mask   device uint8 [B, N], 1 = real token, 0 = padding, or NULL for no padding.  A padded key
+ *             gets score -inf before the softmax (the paper is silent on padding; the graph does not depend
+ *             on the mask).  A padded QUERY row gets out = 0 and lse = -inf.
+ *   out       device, [B, H, N, D], same dtype as q
+ *   lse       device fp32 [B, H, N], natural log of the softmax denominator of each row; may be NULL
+ *   scale     multiplies q.k before the softmax (Eq. (AT) leaves 1/sqrt(d) out; pass it here)
+ *   dtype     BIGBIRD_FP32: fp32 arithmetic on CUDA cores.  BIGBIRD_BF16: tcgen05 tensor-core MMAs with fp32
+ *             accumulation in tensor memory, fp32 softmax, bf16 output.
+ *   stream    cudaStream_t (NULL = default stream).  The call only enqueues work; it never synchronises.
+ *
+ * Supported: D == 64 and b == 64 for BIGBIRD_BF16; D in {32, 64, 128} and any b for BIGBIRD_FP32.
+ * The first call on a device (and the first call with a larger B, N or a new layout) allocates device
+ * scratch owned by the library; later calls allocate nothing.
+ * Errors: BIGBIRD_EINVAL, BIGBIRD_EUNSUPPORTED, BIGBIRD_ECUDA, BIGBIRD_ENOMEM.  There is no CPU path.
+ */
+BIGBIRD_API int bigbird_attn_fwd(const void* q, const void* k, const void* v, const bigbird_layout* layout,
+                     const uint8_t* key_padding_mask, void* out, float* lse,
+                     int B, int H, int64_t N, int D, int b, float scale, int dtype, void* stream);
+
+/*
+ * bigbird_attn_fwd_simt -- the same operation and arguments, always on the CUDA-core kernel (bf16 inputs are
+ * widened to fp32 on load).  A slow, independent GPU path kept for debugging the tensor-core kernel.
+ */
+BIGBIRD_API int bigbird_attn_fwd_simt(const void* q, const void* k, const void* v, const bigbird_layout* layout,
+                          const uint8_t* key_padding_mask, void* out, float* lse,
+                          int B, int H, int64_t N, int D, int b, float scale, int dtype, void* stream);
+
+/*
+ * bigbird_last_status -- synchronises `stream` and reads the device status word of the current device:
+ * BIGBIRD_OK, or BIGBIRD_ETIMEOUT if a bounded wait inside a kernel gave up (the kernel then returned early and
+ * its outputs are invalid).  *detail (may be NULL) receives a code naming the wait.  Clears the word.
+ */
+BIGBIRD_API int bigbird_last_status(void* stream, int* status, int* detail);
+
+/* The cudaError_t of the last failed CUDA call made by the library on this thread (0 if none). */
+BIGBIRD_API int bigbird_last_cuda_error(void);
+
+/* How many kernels the last bigbird_attn_fwd* call on this thread enqueued. */
+BIGBIRD_API int bigbird_last_launch_count(void);
+
+/* A static string for an error code. */
+BIGBIRD_API const char* bigbird_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BIGBIRD_H_ */

@@ -1,0 +1,198 @@
+"""Parity of the CUDA library against the fp64 oracle, through the C-ABI (needs a B200).
+
+Tolerances (max-abs): out 1e-5 for fp32 tensors, 2e-2 for bf16 tensors (fp32 accumulation); lse 1e-3.
+Padded query rows are not compared with the oracle; the library's own contract for them (out = 0,
+lse = -inf) is checked instead.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2007_14062_b200 as bb
+from paper_2007_14062_b200 import synth
+from oracle import bigbird_oracle as O
+
+pytestmark = pytest.mark.gpu
+
+TOL_OUT = {"fp32": 1e-5, "bf16": 2e-2}
+TOL_LSE = 1e-3
+IMPLS = {"fwd": bb.bigbird_attn_fwd, "simt": bb.bigbird_attn_fwd_simt}
+
+
+def _graph(wl):
+    return O.Graph(wl.N, wl.b, wl.w, wl.g, wl.r, wl.seed, wl.H, wl.mode)
+
+
+def _run(wl, q, k, v, kpm, impl="fwd", want_lse=True):
+    dev = torch.device("cuda:0")
+    L = bb.bigbird_build_layout(wl.N, wl.b, wl.w, wl.g, wl.r, wl.seed, wl.H, wl.mode)
+    qd, kd, vd = q.to(dev), k.to(dev), v.to(dev)
+    md = None if kpm is None else kpm.to(dev)
+    out = torch.full_like(qd, float("nan"))
+    lse = torch.full(q.shape[:3], float("nan"), device=dev, dtype=torch.float32) if want_lse else None
+    IMPLS[impl](qd, kd, vd, L, md, out, lse, wl.scale)
+    st, detail = bb.bigbird_last_status()
+    assert st == 0, (st, detail)
+    assert bb.bigbird_last_launch_count() >= 1
+    res = out.float().cpu().numpy(), (None if lse is None else lse.cpu().numpy())
+    L.close()
+    return res
+
+
+def _compare(wl, q, k, v, kpm, out, lse, slices, rows=None):
+    gr = _graph(wl)
+    qn, kn, vn = (t.float().numpy() for t in (q, k, v))      # the exact values handed to the GPU, widened
+    kp = None if kpm is None else kpm.numpy()
+    want = O.attention(qn, kn, vn, gr, kp, wl.scale, slices=slices, rows=rows)
+    rws = np.arange(wl.N) if rows is None else np.asarray(rows)
+    worst_o = worst_l = 0.0
+    for (bi, h), (wo, wlse) in want.items():
+        valid = np.ones(len(rws), dtype=bool) if kp is None else (kp[bi][rws] != 0)
+        go, gl = out[bi, h][rws], lse[bi, h][rws]
+        assert np.isfinite(go).all() and not np.isnan(gl).any()
+        if valid.any():
+            worst_o = max(worst_o, np.abs(go[valid] - wo[valid]).max())
+            worst_l = max(worst_l, np.abs(gl[valid] - wlse[valid]).max())
+        if (~valid).any():                                   # library contract for padded query rows
+            assert (go[~valid] == 0).all() and np.isneginf(gl[~valid]).all()
+    assert worst_o <= TOL_OUT[wl.dtype], (wl.name, worst_o)
+    assert worst_l <= TOL_LSE, (wl.name, worst_l)
+    return worst_o, worst_l
+
+
+def _small(dtype, B, H, nb, lengths="full", mode=0, g=2, r=3, w=3, seed=7, sigma=1.0):
+    return synth.Workload(f"small_{dtype}_{nb}", dtype, B, H, nb * 64, 64, 64, w, g, r, mode, seed=seed, sigma=sigma,
+                          lengths=lengths)
+
+
+# ------------------------------------------------------------------------------------------------ config 1
+@pytest.mark.parametrize("impl", ["fwd", "simt"])
+def test_c1_tiny_itc_fp32_every_element(impl):
+    wl = synth.WORKLOADS["c1_tiny_itc_fp32"]
+    q, k, v = synth.make_qkv(wl)
+    out, lse = _run(wl, q, k, v, None, impl)
+    _compare(wl, q, k, v, None, out, lse, slices=None)
+
+
+# ------------------------------------------------------------------------------------------------ small, several tiles + ragged tails
+SMALL = [
+    _small("bf16", 2, 3, 11),                                   # odd block count: one unpaired tile
+    _small("bf16", 2, 2, 12, lengths="ragged:100:768"),
+    _small("bf16", 1, 2, 9, mode=1, r=0),                       # ETC
+    _small("bf16", 1, 2, 16, g=3, r=2, w=5),
+    _small("bf16", 1, 1, 4, g=4, r=0),                          # every block global
+    _small("bf16", 1, 2, 6, g=0, r=1),                          # no global block
+    _small("bf16", 1, 1, 1, g=1, r=0),                          # a single block
+    _small("fp32", 2, 2, 10, lengths="ragged:64:640"),
+    _small("fp32", 1, 2, 7, mode=1, g=1, r=2),
+]
+
+
+@pytest.mark.parametrize("impl", ["fwd", "simt"])
+@pytest.mark.parametrize("wl", SMALL, ids=lambda w: f"{w.name}_{w.lengths}_{w.mode}_{w.g}{w.r}{w.w}")
+def test_small_cases_every_element(wl, impl):
+    q, k, v = synth.make_qkv(wl)
+    kpm = synth.key_padding_mask(wl)
+    if kpm is not None and wl.B > 1:
+        kpm[1, 197:] = 0            # a length that is not a multiple of the block size
+        kpm[1, :197] = 1
+    out, lse = _run(wl, q, k, v, kpm, impl)
+    _compare(wl, q, k, v, kpm, out, lse, slices=None)
+
+
+@pytest.mark.parametrize("impl", ["fwd", "simt"])
+def test_fully_padded_sequence_and_no_lse(impl):
+    wl = _small("bf16", 2, 2, 8)
+    q, k, v = synth.make_qkv(wl)
+    kpm = torch.ones((2, wl.N), dtype=torch.uint8)
+    kpm[0] = 0                                                    # sequence 0 has no real token at all
+    out, lse = _run(wl, q, k, v, kpm, impl)
+    assert (out[0] == 0).all() and np.isneginf(lse[0]).all()
+    _compare(wl, q, k, v, kpm, out, lse, slices=[(1, 0), (1, 1)])
+    out2, none = _run(wl, q, k, v, kpm, impl, want_lse=False)
+    assert none is None and np.array_equal(out, out2)
+
+
+@pytest.mark.parametrize("impl", ["fwd", "simt"])
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+def test_closed_forms_on_gpu(impl, dtype):
+    """V == 1 gives out == 1; Q == 0 gives lse = ln(#attended valid keys) and out = mean of attended V."""
+    wl = _small(dtype, 1, 2, 12, lengths="fixed:700")
+    q, k, v = synth.make_qkv(wl)
+    kpm = synth.key_padding_mask(wl)
+    out, _ = _run(wl, q, k, torch.ones_like(v), kpm, impl)
+    valid = kpm[0].numpy() != 0
+    assert np.abs(out[0][:, valid] - 1).max() <= (1e-6 if dtype == "fp32" else 2 ** -8)
+    out, lse = _run(wl, torch.zeros_like(q), k, v, kpm, impl)
+    gr = _graph(wl)
+    for h in range(wl.H):
+        A = O.build_mask(gr, h) & valid[None, :]
+        cnt = A.sum(axis=1)
+        assert np.abs(lse[0, h][valid] - np.log(cnt[valid])).max() < 1e-4
+        mean = (A.astype(np.float64) @ v[0, h].double().numpy()) / np.maximum(cnt, 1)[:, None]
+        assert np.abs(out[0, h][valid] - mean[valid]).max() <= TOL_OUT[dtype]
+
+
+def test_two_runs_are_bit_identical():
+    wl = _small("bf16", 2, 4, 16, lengths="ragged:128:1024")
+    q, k, v = synth.make_qkv(wl)
+    kpm = synth.key_padding_mask(wl)
+    a = _run(wl, q, k, v, kpm)
+    b = _run(wl, q, k, v, kpm)
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+
+
+# ------------------------------------------------------------------------------------------------ full-size workloads
+def _sample_slices(wl, n, seed=0):
+    rng = np.random.default_rng(seed)
+    idx = rng.choice(wl.B * wl.H, size=min(n, wl.B * wl.H), replace=False)
+    return sorted((int(i) // wl.H, int(i) % wl.H) for i in idx)
+
+
+def test_c2_base_itc_bf16_full_size():
+    wl = synth.WORKLOADS["c2_base_itc_bf16"]
+    q, k, v = synth.make_qkv(wl)
+    out, lse = _run(wl, q, k, v, None)
+    assert np.isfinite(out).all() and np.isfinite(lse).all()
+    _compare(wl, q, k, v, None, out, lse, slices=_sample_slices(wl, 6) + [(0, 0), (wl.B - 1, wl.H - 1)])
+
+
+def test_c3_etc_bf16_full_size():
+    wl = synth.WORKLOADS["c3_etc_bf16"]
+    q, k, v = synth.make_qkv(wl)
+    out, lse = _run(wl, q, k, v, None)
+    assert np.isfinite(out).all() and np.isfinite(lse).all()
+    _compare(wl, q, k, v, None, out, lse, slices=_sample_slices(wl, 5) + [(0, 0)])
+
+
+def test_c4_long_itc_bf16_full_size():
+    wl = synth.WORKLOADS["c4_long_itc_bf16"]
+    q, k, v = synth.make_qkv(wl)
+    kpm = synth.key_padding_mask(wl)
+    out, lse = _run(wl, q, k, v, kpm)
+    rng = np.random.default_rng(1)
+    rows = np.unique(np.concatenate([
+        np.arange(0, 64), np.arange(wl.N - 64, wl.N),            # the global query blocks (the last one is padding)
+        np.arange(12928, 13056),                                  # around the valid length 13000
+        rng.choice(wl.N, size=320, replace=False)]))
+    _compare(wl, q, k, v, kpm, out, lse, slices=[(0, h) for h in range(0, wl.H, 2)], rows=rows)
+    pad = kpm[0].numpy() == 0
+    assert (out[0][:, pad] == 0).all() and np.isneginf(lse[0][:, pad]).all()
+    assert np.isfinite(out).all() and np.isfinite(lse[0][:, ~pad]).all()
+
+
+def test_c5_large_ragged_bf16_full_size():
+    wl = synth.WORKLOADS["c5_large_ragged_bf16"]
+    q, k, v = synth.make_qkv(wl)
+    kpm = synth.key_padding_mask(wl)
+    lens = synth.valid_lengths(wl)
+    out, lse = _run(wl, q, k, v, kpm)
+    shortest, longest = int(np.argmin(lens)), int(np.argmax(lens))
+    slices = sorted(set([(shortest, 0), (shortest, wl.H - 1), (longest, 3), (longest, 8)] + _sample_slices(wl, 4, seed=2)))
+    _compare(wl, q, k, v, kpm, out, lse, slices=slices)
+    assert np.isfinite(out).all()
+    for bi in range(wl.B):
+        assert (out[bi][:, lens[bi]:] == 0).all() and np.isneginf(lse[bi][:, lens[bi]:]).all()
+        assert np.isfinite(lse[bi][:, : lens[bi]]).all()
