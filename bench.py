@@ -1,0 +1,325 @@
+#!/usr/bin/env python
+"""Benchmark of the BigBird block-sparse attention forward pass on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+One "step" is one pass of the whole hot path (layout already built; Q/K/V -> out, lse) over one batch of
+the BigBird-base workload: B=8, H=12, N=4096, D=64, block 64, 3 window + 2 global + 3 random blocks, bf16.
+The metric counts only the FLOPs of the attended block pairs (4*b*b*D each).  Rank 0 prints one JSON line.
+
+With N > 1 (under torchrun) every rank runs the same workload on its own GPU (the op shards over batch and
+head with no exchange, so there is no collective on the data path); the value is the total over ranks
+divided by the slowest rank's time.
+
+`--impl reference` times the fp64 CPU oracle as it stands on the host cores (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2007_14062_b200 import synth  # noqa: E402
+
+METRIC = "block-sparse attn fwd TFLOP/s (counted FLOPs) & % bf16 TC peak at N=4096"
+UNIT = "TFLOP/s"
+NOMINAL_BF16_TFLOPS = 2250.0
+FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "hbm_gbs": 6650.0}
+# dram__bytes_read.sum + dram__bytes_write.sum of one attn_fwd_sm100_kernel launch on this workload, from the
+# ncu capture summarised in profiles/ (None until a capture exists for the current kernel).
+NCU_DRAM_BYTES_PER_LAUNCH = {"c2_base_itc_bf16": None}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"bf16_tflops": float(d["bf16_tflops"]), "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", 0)),
+                "hbm_gbs": float(d["hbm_gbs"]), "source": "measured"}
+    return dict(FALLBACK_PEAKS, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+def counted_pairs(layout, wl) -> int:
+    """Attended (query block, key block) pairs per batch element, summed over heads."""
+    return int(layout.nnz)
+
+
+class ClockSampler:
+    """Samples SM clock and clock-event reasons of the benchmarked GPU through NVML while the timed region runs."""
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting", 0x10: "sync_boost"}
+
+    def __init__(self, device_index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode() if hasattr(uuid, "encode") else uuid)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception as e:  # NVML missing: report that no clocks were sampled
+            self.nv, self.h, self.err = None, None, repr(e)
+
+    def _loop(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                bits = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in self.REASONS.items():
+                    if bits & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def oracle_slices(wl, q, k, v, kpm, slices):
+    from oracle import bigbird_oracle as O
+    gr = O.Graph(wl.N, wl.b, wl.w, wl.g, wl.r, wl.seed, wl.H, wl.mode)
+    t0 = time.perf_counter()
+    O.attention(q, k, v, gr, kpm, wl.scale, slices=slices)
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(wl, pairs_per_batch, budget_s=12.0):
+    """Times the oracle, as it stands, on a bounded sample of (batch, head) slices of the workload."""
+    q, k, v = synth.make_qkv(wl, batch_limit=1)
+    qn, kn, vn = (t.float().numpy() for t in (q, k, v))
+    kpm = synth.key_padding_mask(wl)
+    kp = None if kpm is None else kpm.numpy()
+    flops_per_slice = pairs_per_batch / wl.H * 4.0 * wl.b * wl.b * wl.D
+    t1 = oracle_slices(wl, qn, kn, vn, kp, [(0, 0)])
+    n = int(max(1, min(wl.H - 1, budget_s / max(t1, 1e-3))))
+    slices = [(0, 1 + i) for i in range(n)] if wl.H > 1 else [(0, 0)]
+    t = oracle_slices(wl, qn, kn, vn, kp, slices)
+    cores = len(os.sched_getaffinity(0))
+    return {"value": flops_per_slice * len(slices) / t / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{len(slices)} of {wl.B * wl.H} (batch, head) slices at full N={wl.N}, fp64 masked dense attention; "
+                      f"{t / len(slices):.3f} s per slice",
+            "seconds_per_slice": t / len(slices)}
+
+
+def run_reference(args, wl):
+    """The oracle as the reference arm: each step is one (batch, head) slice at full sequence length."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import paper_2007_14062_b200 as bb
+    L = bb.bigbird_build_layout(wl.N, wl.b, wl.w, wl.g, wl.r, wl.seed, wl.H, wl.mode)
+    flops_per_slice = counted_pairs(L, wl) / wl.H * 4.0 * wl.b * wl.b * wl.D
+    q, k, v = synth.make_qkv(wl, batch_limit=1)
+    qn, kn, vn = (t.float().numpy() for t in (q, k, v))
+    kpm = synth.key_padding_mask(wl)
+    kp = None if kpm is None else kpm.numpy()
+    for i in range(args.warmup):
+        oracle_slices(wl, qn, kn, vn, kp, [(0, i % wl.H)])
+    t = 0.0
+    for i in range(args.steps):
+        t += oracle_slices(wl, qn, kn, vn, kp, [(0, i % wl.H)])
+    value = flops_per_slice * args.steps / t / 1e12
+    cores = len(os.sched_getaffinity(0))
+    sample = f"each step = 1 of {wl.B * wl.H} (batch, head) slices at full N={wl.N} (fp64 masked dense attention on the host)"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "N": wl.N, "D": wl.D, "block": wl.b, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3000)
+    ap.add_argument("--warmup", type=int, default=50)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2_base_itc_bf16", choices=synth.ORDER)
+    ap.add_argument("--e2e-steps", type=int, default=20)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    wl = synth.WORKLOADS[args.workload]
+
+    if args.impl == "reference":
+        if args.steps == 3000:
+            args.steps, args.warmup = 12, 3
+        run_reference(args, wl)
+        return
+    if args.warmup < 3:
+        args.warmup = 3
+
+    import paper_2007_14062_b200 as bb
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    L = bb.bigbird_build_layout(wl.N, wl.b, wl.w, wl.g, wl.r, wl.seed, wl.H, wl.mode)
+    pairs = counted_pairs(L, wl)
+    flops_per_step = wl.B * pairs * 4.0 * wl.b * wl.b * wl.D
+    tokens_per_step = wl.B * wl.N
+
+    # Rotating input sets so that no step finds its inputs in L2 (4 sets x 201 MB for the base workload; L2 is 126 MB).
+    q, k, v = synth.make_qkv(wl)
+    kpm = synth.key_padding_mask(wl)
+    n_sets = 4
+    sets = []
+    for i in range(n_sets):
+        qd, kd, vd = (t.to(dev) for t in (q, k, v))
+        if i:
+            qd, kd, vd = qd.roll(i, 0), kd.roll(i, 0), vd.roll(i, 0)          # same values, other batch order
+        md = None if kpm is None else kpm.roll(i, 0).to(dev).contiguous()
+        sets.append((qd.contiguous(), kd.contiguous(), vd.contiguous(), md, torch.empty_like(qd),
+                     torch.empty(q.shape[:3], device=dev, dtype=torch.float32)))
+    stream = torch.cuda.current_stream(dev)
+
+    def step(i):
+        qd, kd, vd, md, od, ld = sets[i % n_sets]
+        bb.bigbird_attn_fwd(qd, kd, vd, L, md, od, ld, wl.scale, stream.cuda_stream)
+
+    for i in range(args.warmup):
+        step(i)
+    launches_per_step = bb.bigbird_last_launch_count()
+    st, detail = bb.bigbird_last_status(stream.cuda_stream)
+    if st != 0:
+        raise SystemExit(f"kernel reported status {st} (wait {detail})")
+
+    sampler = ClockSampler(local_rank)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    sampler.start()
+    ev0.record(stream)
+    for i in range(args.steps):
+        step(i)
+    ev1.record(stream)
+    barrier()
+    sampler.stop()
+    ms = ev0.elapsed_time(ev1)
+    st, detail = bb.bigbird_last_status(stream.cuda_stream)
+    if st != 0:
+        raise SystemExit(f"kernel reported status {st} (wait {detail})")
+
+    # ---- end to end: pinned host buffers in, results back to the host, every step ----
+    hq, hk, hv = (t.pin_memory() for t in (q, k, v))
+    hm = None if kpm is None else kpm.pin_memory()
+    ho = torch.empty_like(q).pin_memory()
+    hl = torch.empty(q.shape[:3], dtype=torch.float32).pin_memory()
+    dq, dk, dv, dm, do, dl_ = sets[0]
+
+    def e2e_step():
+        dq.copy_(hq, non_blocking=True)
+        dk.copy_(hk, non_blocking=True)
+        dv.copy_(hv, non_blocking=True)
+        if hm is not None:
+            dm.copy_(hm, non_blocking=True)
+        bb.bigbird_attn_fwd(dq, dk, dv, L, dm, do, dl_, wl.scale, stream.cuda_stream)
+        ho.copy_(do, non_blocking=True)
+        hl.copy_(dl_, non_blocking=True)
+
+    for _ in range(3):
+        e2e_step()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for _ in range(args.e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv)) + (0 if hm is None else hm.numel())
+    d2h = ho.numel() * ho.element_size() + hl.numel() * 4
+
+    if dist is not None:
+        t = torch.tensor([ms, e2e_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, e2e_ms = float(t[0]), float(t[1])
+
+    if rank == 0:
+        peaks = measured_peaks()
+        ms_per_step = ms / args.steps
+        tflops = world * flops_per_step / (ms_per_step * 1e-3) / 1e12
+        per_gpu = tflops / world
+        e2e_tflops = world * flops_per_step / (e2e_ms / args.e2e_steps * 1e-3) / 1e12
+        traffic = NCU_DRAM_BYTES_PER_LAUNCH.get(wl.name)
+        min_bytes = wl.B * wl.H * wl.N * (4 * wl.D * 2 + 4)
+        line = {
+            "metric": METRIC, "value": tflops, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "N": wl.N, "D": wl.D, "block": wl.b, "window_blocks": wl.w,
+                       "global_blocks": wl.g, "random_blocks": wl.r, "mode": "ETC" if wl.mode else "ITC",
+                       "attended_block_pairs_per_step": wl.B * pairs, "counted_gflop_per_step": flops_per_step / 1e9,
+                       "l2": f"rotating {n_sets} input/output sets ({n_sets * 4 * q.numel() * 2 / 1e6:.0f} MB) larger than L2",
+                       "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
+            "tokens_per_s": world * tokens_per_step / (ms_per_step * 1e-3),
+            "pct_of_measured_bf16_peak": 100.0 * per_gpu / peaks["bf16_tflops"],
+            "pct_of_nominal_bf16_peak": 100.0 * per_gpu / NOMINAL_BF16_TFLOPS,
+            "e2e": {"value": e2e_tflops, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "steps": args.e2e_steps, "ms_per_step": e2e_ms / args.e2e_steps},
+            "gpu_launches": launches_per_step * args.steps,
+            "clocks": sampler.summary(),
+            "roofline": {"bound": "tensor", "achieved": per_gpu, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                         "frac": per_gpu / peaks["bf16_tflops"], "traffic": traffic,
+                         "peak_source": f"{peaks['source']} bf16 burst", "kernel": "attn_fwd_sm100_kernel",
+                         "kernel_us": 1e3 * ms_per_step, "algorithmic_flops_per_launch": flops_per_step,
+                         "min_hbm_bytes_per_launch": min_bytes,
+                         "achieved_hbm_gbs_on_min_bytes": min_bytes / (ms_per_step * 1e-3) / 1e9,
+                         "frac_of_sustained_peak": per_gpu / peaks["bf16_tflops_sustained"] if peaks["bf16_tflops_sustained"] else None},
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(wl, pairs)
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
