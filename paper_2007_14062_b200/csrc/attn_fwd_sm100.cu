@@ -33,24 +33,50 @@ namespace {
 constexpr int kBlock = 64;                 // tokens per block (b) and head dimension (D)
 constexpr int kTileBytes = kBlock * kBlock * 2;      // one 64x64 bf16 tile
 constexpr int kRingSlots = 10;
-constexpr int kThreads = 192;              // warp 0 producer, warp 1 MMA issuer, warps 2..5 softmax
+constexpr int kThreads = 256;              // warp 0 TMA, warp 1 MMA issuer, warp 2 scheduler, warp 3 idle, warps 4..7 softmax
 constexpr int kSoftmaxWarps = 4;
+#ifndef BB_REGS_LIGHT
+#define BB_REGS_LIGHT 64
+#define BB_REGS_SOFTMAX 192
+#endif
+constexpr int kRegsLight = BB_REGS_LIGHT;             // registers per thread of warps 0..3 after setmaxnreg
+constexpr int kRegsSoftmax = BB_REGS_SOFTMAX;          // registers per thread of warps 4..7 after setmaxnreg
 constexpr int kTmemCols = 256;
 constexpr int kColS = 0;                   // scores: 2 x 64 fp32 columns
 constexpr int kColP = 128;                 // probabilities: 2 x 32 columns of packed bf16 pairs
 constexpr int kColO = 192;                 // output accumulator: 64 fp32 columns
 constexpr float kRescaleThreshold = 8.0f;  // in log2 units
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+constexpr int kSchedSlots = 3;
+constexpr int kSegSteps = 64;              // live steps per posted segment of a tile
 
-struct __align__(8) SmemCtl {
+// A step of a tile after the key-padding mask has been applied: key blocks that are entirely padding are gone.
+struct __align__(16) StepEntry {
+    int c0, c1;                    // key block of the upper / lower half (or of both when full), -1 = none
+    int full;
+    int pad_;
+    unsigned long long kb0, kb1;   // valid-key bits of c0 / c1
+};
+enum { kSegFirst = 1, kSegLast = 2, kSegLive = 4 };
+struct __align__(16) WorkSlot {
+    int w;                         // work index, -1 = no more work
+    int bh, batch, qa, qb;
+    int n_steps;
+    int flags;
+    int pad_;
+    unsigned long long qbits_a, qbits_b;
+    StepEntry steps[kSegSteps];
+};
+
+struct __align__(16) SmemCtl {
     unsigned long long full[kRingSlots];
     unsigned long long empty[kRingSlots];
     unsigned long long q_full, q_empty;
     unsigned long long s_full, s_free, p_full, pv_done;
-    unsigned long long sched_full[2], sched_empty[2];
-    int work[2];
+    unsigned long long sched_full[kSchedSlots], sched_empty[kSchedSlots];
     unsigned tmem_base;
     int abort_flag;
+    WorkSlot slot[kSchedSlots];
 };
 constexpr int kSmemQ = 0;
 constexpr int kSmemRing = 2 * kTileBytes;
@@ -99,7 +125,7 @@ __device__ __forceinline__ unsigned long long global_ns() {
 }
 
 // Bounded wait.  Returns false if the wait expired or another thread of the CTA already gave up.
-__device__ __noinline__ bool mbar_wait_slow(unsigned long long* bar, unsigned parity, SmemCtl* ctl, int* status, int code) {
+__device__ __forceinline__ bool mbar_wait_slow(unsigned long long* bar, unsigned parity, SmemCtl* ctl, int* status, int code) {
     const unsigned long long t0 = global_ns();
     for (unsigned it = 0;; ++it) {
         if (mbar_try(bar, parity)) return true;
@@ -156,36 +182,38 @@ __device__ __forceinline__ unsigned long long smem_desc_sw128(unsigned addr) {
 constexpr unsigned kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
 constexpr unsigned kIdescPV = kIdescQK | (1u << 16);
 
+#define BB_REP32(F, o) F(o+0), F(o+1), F(o+2), F(o+3), F(o+4), F(o+5), F(o+6), F(o+7), F(o+8), F(o+9), F(o+10), F(o+11), \
+    F(o+12), F(o+13), F(o+14), F(o+15), F(o+16), F(o+17), F(o+18), F(o+19), F(o+20), F(o+21), F(o+22), F(o+23), \
+    F(o+24), F(o+25), F(o+26), F(o+27), F(o+28), F(o+29), F(o+30), F(o+31)
+#define BB_OUT(i) "=r"(u[i])
+#define BB_IN(i) "r"(u[i])
 __device__ __forceinline__ void tmem_ld64(unsigned taddr, float* r) {
     unsigned* u = reinterpret_cast<unsigned*>(r);
-#define BB_R(i) "=r"(u[i])
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x64.b32 "
         "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
         "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, "
         "%32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, "
         "%48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];"
-        : BB_R(0), BB_R(1), BB_R(2), BB_R(3), BB_R(4), BB_R(5), BB_R(6), BB_R(7), BB_R(8), BB_R(9), BB_R(10), BB_R(11),
-          BB_R(12), BB_R(13), BB_R(14), BB_R(15), BB_R(16), BB_R(17), BB_R(18), BB_R(19), BB_R(20), BB_R(21), BB_R(22),
-          BB_R(23), BB_R(24), BB_R(25), BB_R(26), BB_R(27), BB_R(28), BB_R(29), BB_R(30), BB_R(31), BB_R(32), BB_R(33),
-          BB_R(34), BB_R(35), BB_R(36), BB_R(37), BB_R(38), BB_R(39), BB_R(40), BB_R(41), BB_R(42), BB_R(43), BB_R(44),
-          BB_R(45), BB_R(46), BB_R(47), BB_R(48), BB_R(49), BB_R(50), BB_R(51), BB_R(52), BB_R(53), BB_R(54), BB_R(55),
-          BB_R(56), BB_R(57), BB_R(58), BB_R(59), BB_R(60), BB_R(61), BB_R(62), BB_R(63)
-        : "r"(taddr) : "memory");
-#undef BB_R
+        : BB_REP32(BB_OUT, 0), BB_REP32(BB_OUT, 32) : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(unsigned taddr, float* r) {
+    unsigned* u = reinterpret_cast<unsigned*>(r);
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : BB_REP32(BB_OUT, 0) : "r"(taddr) : "memory");
 }
 __device__ __forceinline__ void tmem_st32(unsigned taddr, const unsigned* u) {
-#define BB_R(i) "r"(u[i])
     asm volatile(
         "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
         "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
         "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31};"
-        ::BB_R(0), BB_R(1), BB_R(2), BB_R(3), BB_R(4), BB_R(5), BB_R(6), BB_R(7), BB_R(8), BB_R(9), BB_R(10), BB_R(11),
-          BB_R(12), BB_R(13), BB_R(14), BB_R(15), BB_R(16), BB_R(17), BB_R(18), BB_R(19), BB_R(20), BB_R(21), BB_R(22),
-          BB_R(23), BB_R(24), BB_R(25), BB_R(26), BB_R(27), BB_R(28), BB_R(29), BB_R(30), BB_R(31), "r"(taddr)
-        : "memory");
-#undef BB_R
+        ::BB_REP32(BB_IN, 0), "r"(taddr) : "memory");
 }
+#undef BB_OUT
+#undef BB_IN
 __device__ __forceinline__ void tmem_st32_zero(unsigned taddr) {
     const unsigned z = 0;
     asm volatile(
@@ -207,51 +235,30 @@ __device__ __forceinline__ unsigned pack_bf16(float lo, float hi) {
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
     return d;
 }
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+// (x0, x1) * a + b on the packed fp32 pipe
+__device__ __forceinline__ void ffma2(float& r0, float& r1, float x0, float x1, float a, float b) {
+    asm("{ .reg .b64 ra, rb, rc, rd; mov.b64 ra, {%2, %3}; mov.b64 rb, {%4, %4}; mov.b64 rc, {%5, %5}; "
+        "fma.rn.f32x2 rd, ra, rb, rc; mov.b64 {%0, %1}, rd; }"
+        : "=f"(r0), "=f"(r1) : "f"(x0), "f"(x1), "f"(a), "f"(b));
+}
+__device__ __forceinline__ void fadd2(float& r0, float& r1, float x0, float x1) {
+    asm("{ .reg .b64 ra, rb, rd; mov.b64 ra, {%0, %1}; mov.b64 rb, {%2, %3}; add.f32x2 rd, ra, rb; mov.b64 {%0, %1}, rd; }"
+        : "+f"(r0), "+f"(r1) : "f"(x0), "f"(x1));
+}
+__device__ __forceinline__ void fmul2(float& r0, float& r1, float a) {
+    asm("{ .reg .b64 ra, rb, rd; mov.b64 ra, {%0, %1}; mov.b64 rb, {%2, %2}; mul.f32x2 rd, ra, rb; mov.b64 {%0, %1}, rd; }"
+        : "+f"(r0), "+f"(r1) : "f"(a));
+}
 
 // ------------------------------------------------------------------------------------------------ schedule helpers
-struct Work {
-    int bh, h, batch;
-    Item item;
-};
-__device__ __forceinline__ Work decode_work(const KernelParams& p, int w) {
-    Work k;
-    int it;
-    const int heavy_total = p.BH * p.heavy_per_head;
-    if (w < heavy_total) {
-        k.bh = w / p.heavy_per_head;
-        it = w - k.bh * p.heavy_per_head;
-    } else {
-        const int sparse = p.items_per_head - p.heavy_per_head;
-        const int w2 = w - heavy_total;
-        k.bh = w2 / sparse;
-        it = p.heavy_per_head + (w2 - k.bh * sparse);
-    }
-    k.h = k.bh % p.H;
-    k.batch = k.bh / p.H;
-    k.item = p.items[(size_t)k.h * p.items_per_head + it];
-    return k;
-}
 __device__ __forceinline__ unsigned long long key_bits(const KernelParams& p, int batch, int c) {
     if (c < 0) return 0ull;
     return p.kbits ? p.kbits[(size_t)batch * p.nb + c] : ~0ull;
-}
-// Key blocks of a step that take part: (c0 or -1, c1 or -1); full step: c1 = kStepFull.
-struct LiveStep {
-    int c0, c1;
-    bool full;
-    __device__ bool any() const { return c0 >= 0 || c1 >= 0; }
-};
-__device__ __forceinline__ LiveStep live_step(const KernelParams& p, int batch, Step s, bool has_qb) {
-    LiveStep l;
-    l.full = s.c1 == kStepFull;
-    l.c0 = key_bits(p, batch, s.c0) ? s.c0 : -1;
-    l.c1 = (!l.full && has_qb && key_bits(p, batch, s.c1)) ? s.c1 : -1;
-    return l;
-}
-// A tile is skipped when none of its query rows is a real token.
-__device__ __forceinline__ bool tile_is_live(const KernelParams& p, const Work& w) {
-    if (!p.kbits) return true;
-    return (key_bits(p, w.batch, w.item.qa) | key_bits(p, w.batch, w.item.qb)) != 0ull;
 }
 
 // ------------------------------------------------------------------------------------------------ the kernel
@@ -271,7 +278,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         mbar_init(&ctl->s_free, kSoftmaxWarps);
         mbar_init(&ctl->p_full, kSoftmaxWarps);
         mbar_init(&ctl->pv_done, 1);
-        for (int i = 0; i < 2; ++i) { mbar_init(&ctl->sched_full[i], 1); mbar_init(&ctl->sched_empty[i], 1 + kSoftmaxWarps); }
+        for (int i = 0; i < kSchedSlots; ++i) { mbar_init(&ctl->sched_full[i], 1); mbar_init(&ctl->sched_empty[i], 2 + kSoftmaxWarps); }
         ctl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -285,9 +292,86 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     tc_fence_after();
     const unsigned tmem = *(volatile unsigned*)&ctl->tmem_base;
 
-    if (warp == 0) {
-        // ===================================================================== producer: scheduler + TMA
-        if (lane == 0) {
+    if (warp < 4) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsLight));
+        if (warp == 2) {
+            // ================================================================= scheduler: fetch work, post live steps
+            unsigned sched_n = 0;
+            bool ok = true;
+            const unsigned lt_mask = (1u << lane) - 1u;
+            while (ok) {
+                int w = 0;
+                if (lane == 0) w = atomicAdd(&p.counter[0], 1);
+                w = __shfl_sync(0xffffffffu, w, 0);
+                if (w >= p.total_work) w = -1;
+                // decode the work index: global-row tiles of every (batch, head) first, then the sparse tiles
+                int bh = 0, it = 0;
+                Item item{};
+                if (w >= 0) {
+                    const int heavy_total = p.BH * p.heavy_per_head;
+                    if (w < heavy_total) {
+                        bh = w / p.heavy_per_head;
+                        it = w - bh * p.heavy_per_head;
+                    } else {
+                        const int sparse = p.items_per_head - p.heavy_per_head;
+                        const int w2 = w - heavy_total;
+                        bh = w2 / sparse;
+                        it = p.heavy_per_head + (w2 - bh * sparse);
+                    }
+                    item = p.items[(size_t)(bh % p.H) * p.items_per_head + it];
+                }
+                const int batch = bh / p.H;
+                const bool has_qb = item.qb >= 0;
+                const unsigned long long qbits_a = w >= 0 ? key_bits(p, batch, item.qa) : 0ull;
+                const unsigned long long qbits_b = w >= 0 ? key_bits(p, batch, item.qb) : 0ull;
+                const bool tile_live = (qbits_a | qbits_b) != 0ull;      // a tile whose query rows are all padding is skipped
+                const int n_raw = (w >= 0 && tile_live) ? item.step_count : 0;
+                int i0 = 0;
+                bool first = true;
+                do {
+                    const unsigned ss = sched_n % kSchedSlots, sp = (sched_n / kSchedSlots) & 1u;
+                    ok = mbar_wait(&ctl->sched_empty[ss], sp ^ 1u, ctl, p.status, 11);
+                    if (!ok) break;
+                    WorkSlot* slot = &ctl->slot[ss];
+                    int count = 0;
+                    while (i0 < n_raw && count <= kSegSteps - 32) {
+                        const int i = i0 + lane;
+                        StepEntry e{-1, -1, 0, 0, 0ull, 0ull};
+                        if (i < n_raw) {
+                            const Step s = p.steps[item.step_begin + i];
+                            e.full = s.c1 == kStepFull;
+                            e.kb0 = key_bits(p, batch, s.c0);
+                            e.kb1 = (!e.full && has_qb) ? key_bits(p, batch, s.c1) : 0ull;
+                            e.c0 = e.kb0 ? s.c0 : -1;
+                            e.c1 = e.kb1 ? s.c1 : -1;
+                        }
+                        const bool alive = e.c0 >= 0 || e.c1 >= 0;
+                        const unsigned bal = __ballot_sync(0xffffffffu, alive);
+                        if (alive) slot->steps[count + __popc(bal & lt_mask)] = e;
+                        count += __popc(bal);
+                        i0 += 32;
+                    }
+                    if (lane == 0) {
+                        slot->w = w;
+                        slot->bh = bh;
+                        slot->batch = batch;
+                        slot->qa = item.qa;
+                        slot->qb = item.qb;
+                        slot->n_steps = count;
+                        slot->flags = (first ? kSegFirst : 0) | (i0 >= n_raw ? kSegLast : 0) | (tile_live ? kSegLive : 0);
+                        slot->qbits_a = qbits_a;
+                        slot->qbits_b = qbits_b;
+                    }
+                    __threadfence_block();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&ctl->sched_full[ss]);
+                    ++sched_n;
+                    first = false;
+                } while (i0 < n_raw);
+                if (w < 0) break;
+            }
+        } else if (warp == 0 && lane == 0) {
+            // ================================================================= TMA producer
             unsigned ring_n = 0, q_n = 0, sched_n = 0;
             bool ok = true;
             auto load = [&](const CUtensorMap* tm, int bh, int block) -> bool {
@@ -298,46 +382,45 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                 ++ring_n;
                 return true;
             };
-            auto load_step = [&](const CUtensorMap* tm, int bh, const LiveStep& l) -> bool {
-                if (l.c0 >= 0 && !load(tm, bh, l.c0)) return false;
-                if (l.c1 >= 0 && !load(tm, bh, l.c1)) return false;
+            auto load_pair = [&](const CUtensorMap* tm, int bh, int c0, int c1) -> bool {
+                if (c0 >= 0 && !load(tm, bh, c0)) return false;
+                if (c1 >= 0 && !load(tm, bh, c1)) return false;
                 return true;
             };
+            int prev_c0 = -1, prev_c1 = -1;
             while (ok) {
-                int w = atomicAdd(&p.counter[0], 1);
-                if (w >= p.total_work) w = -1;
-                const unsigned ss = sched_n & 1u, sp = (sched_n >> 1) & 1u;
-                if (!mbar_wait(&ctl->sched_empty[ss], sp ^ 1u, ctl, p.status, 11)) break;
-                ctl->work[ss] = w;
-                mbar_arrive(&ctl->sched_full[ss]);      // arrive has release semantics: the store above is visible
+                const unsigned ss = sched_n % kSchedSlots, sp = (sched_n / kSchedSlots) & 1u;
+                if (!mbar_wait(&ctl->sched_full[ss], sp, ctl, p.status, 13)) break;
+                const WorkSlot* slot = &ctl->slot[ss];
+                const int w = slot->w, flags = slot->flags, bh = slot->bh, n = slot->n_steps;
+                if (w >= 0 && (flags & kSegLive)) {
+                    if (flags & kSegFirst) {
+                        const int qa = slot->qa, qb = slot->qb;
+                        ok = mbar_wait(&ctl->q_empty, (q_n & 1u) ^ 1u, ctl, p.status, 12);
+                        if (!ok) break;
+                        mbar_expect_tx(&ctl->q_full, qb >= 0 ? 2 * kTileBytes : kTileBytes);
+                        tma_load_tile(smem + kSmemQ, &tm_q, (bh * p.nb + qa) * kBlock, &ctl->q_full);
+                        if (qb >= 0) tma_load_tile(smem + kSmemQ + kTileBytes, &tm_q, (bh * p.nb + qb) * kBlock, &ctl->q_full);
+                        ++q_n;
+                        prev_c0 = prev_c1 = -1;
+                    }
+                    // K of step i+1 goes ahead of V of step i: the order in which the MMA thread consumes them
+                    for (int i = 0; i < n && ok; ++i) {
+                        const int c0 = slot->steps[i].c0, c1 = slot->steps[i].c1;
+                        ok = load_pair(&tm_k, bh, c0, c1);
+                        if (ok) ok = load_pair(&tm_v, bh, prev_c0, prev_c1);
+                        prev_c0 = c0;
+                        prev_c1 = c1;
+                    }
+                    if (ok && (flags & kSegLast)) ok = load_pair(&tm_v, bh, prev_c0, prev_c1);
+                }
+                mbar_arrive(&ctl->sched_empty[ss]);
                 ++sched_n;
                 if (w < 0) break;
-                const Work wk = decode_work(p, w);
-                if (!tile_is_live(p, wk)) continue;
-                const bool has_qb = wk.item.qb >= 0;
-                // Q tile(s)
-                if (!mbar_wait(&ctl->q_empty, (q_n & 1u) ^ 1u, ctl, p.status, 12)) break;
-                mbar_expect_tx(&ctl->q_full, has_qb ? 2 * kTileBytes : kTileBytes);
-                tma_load_tile(smem + kSmemQ, &tm_q, (wk.bh * p.nb + wk.item.qa) * kBlock, &ctl->q_full);
-                if (has_qb) tma_load_tile(smem + kSmemQ + kTileBytes, &tm_q, (wk.bh * p.nb + wk.item.qb) * kBlock, &ctl->q_full);
-                ++q_n;
-                // K of step i+1 goes ahead of V of step i: the order in which the MMA thread consumes them
-                LiveStep prev{-1, -1, false};
-                for (int i = 0; i < wk.item.step_count && ok; ++i) {
-                    const LiveStep l = live_step(p, wk.batch, p.steps[wk.item.step_begin + i], has_qb);
-                    if (!l.any()) continue;
-                    ok = load_step(&tm_k, wk.bh, l);
-                    if (ok && prev.any()) ok = load_step(&tm_v, wk.bh, prev);
-                    prev = l;
-                }
-                if (ok && prev.any()) ok = load_step(&tm_v, wk.bh, prev);
             }
-        }
-    } else if (warp == 1) {
-        // ===================================================================== MMA issuer
-        if (lane == 0) {
-            unsigned ring_n = 0, q_n = 0, sched_n = 0, grp_n = 0;     // grp_n: live steps issued so far (QK groups)
-            unsigned pv_n = 0;
+        } else if (warp == 1 && lane == 0) {
+            // ================================================================= MMA issuer
+            unsigned ring_n = 0, q_n = 0, sched_n = 0, grp_n = 0, pv_n = 0;   // grp_n: live steps whose Q K^T was issued
             bool ok = true;
             const unsigned long long q_desc = smem_desc_sw128(smem_u32(smem + kSmemQ));
             auto qk = [&](int col_off) -> bool {        // S[:, col_off .. col_off+63] = Q K^T with K in the next ring slot
@@ -364,180 +447,208 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                 ++ring_n;
                 return true;
             };
-            auto pv_step = [&](const LiveStep& l) -> bool {
+            auto pv_step = [&](int c0, int c1) -> bool {
                 if (!mbar_wait(&ctl->p_full, pv_n & 1u, ctl, p.status, 22)) return false;
                 tc_fence_after();
-                if (l.c0 >= 0 && !pv(0)) return false;
-                if (l.c1 >= 0 && !pv(32)) return false;
+                if (c0 >= 0 && !pv(0)) return false;
+                if (c1 >= 0 && !pv(32)) return false;
                 tc_commit(&ctl->pv_done);
                 ++pv_n;
                 return true;
             };
+            int prev_c0 = -1, prev_c1 = -1;
             while (ok) {
-                const unsigned ss = sched_n & 1u, sp = (sched_n >> 1) & 1u;
+                const unsigned ss = sched_n % kSchedSlots, sp = (sched_n / kSchedSlots) & 1u;
                 if (!mbar_wait(&ctl->sched_full[ss], sp, ctl, p.status, 23)) break;
-                const int w = *(volatile int*)&ctl->work[ss];
+                const WorkSlot* slot = &ctl->slot[ss];
+                const int w = slot->w, flags = slot->flags, n = slot->n_steps;
+                if (w >= 0 && (flags & kSegLive)) {
+                    if (flags & kSegFirst) {
+                        ok = mbar_wait(&ctl->q_full, q_n & 1u, ctl, p.status, 24);
+                        if (!ok) break;
+                        tc_fence_after();
+                        prev_c0 = prev_c1 = -1;
+                    }
+                    for (int i = 0; i < n && ok; ++i) {
+                        const int c0 = slot->steps[i].c0, c1 = slot->steps[i].c1;
+                        // the softmax warps must have pulled the previous scores out of tensor memory
+                        ok = mbar_wait(&ctl->s_free, (grp_n & 1u) ^ 1u, ctl, p.status, 25);
+                        if (!ok) break;
+                        tc_fence_after();
+                        if (c0 >= 0) ok = qk(0);
+                        if (ok && c1 >= 0) ok = qk(64);
+                        if (!ok) break;
+                        tc_commit(&ctl->s_full);
+                        ++grp_n;
+                        if (prev_c0 >= 0 || prev_c1 >= 0) ok = pv_step(prev_c0, prev_c1);
+                        prev_c0 = c0;
+                        prev_c1 = c1;
+                    }
+                    if (!ok) break;
+                    if (flags & kSegLast) {
+                        tc_commit(&ctl->q_empty);       // every Q K^T of the tile has been issued
+                        ++q_n;
+                        if (prev_c0 >= 0 || prev_c1 >= 0) ok = pv_step(prev_c0, prev_c1);
+                    }
+                }
                 mbar_arrive(&ctl->sched_empty[ss]);
                 ++sched_n;
                 if (w < 0) break;
-                const Work wk = decode_work(p, w);
-                if (!tile_is_live(p, wk)) continue;
-                const bool has_qb = wk.item.qb >= 0;
-                if (!mbar_wait(&ctl->q_full, q_n & 1u, ctl, p.status, 24)) break;
-                tc_fence_after();
-                LiveStep prev{-1, -1, false};
-                for (int i = 0; i < wk.item.step_count && ok; ++i) {
-                    const LiveStep l = live_step(p, wk.batch, p.steps[wk.item.step_begin + i], has_qb);
-                    if (!l.any()) continue;
-                    // the softmax warps must have pulled the previous scores out of tensor memory
-                    ok = mbar_wait(&ctl->s_free, (grp_n & 1u) ^ 1u, ctl, p.status, 25);
-                    if (!ok) break;
-                    tc_fence_after();
-                    if (l.c0 >= 0) ok = qk(0);
-                    if (ok && l.c1 >= 0) ok = qk(64);
-                    if (!ok) break;
-                    tc_commit(&ctl->s_full);
-                    ++grp_n;
-                    if (prev.any()) ok = pv_step(prev);
-                    prev = l;
-                }
-                if (!ok) break;
-                tc_commit(&ctl->q_empty);               // every Q K^T of the tile has been issued
-                ++q_n;
-                if (prev.any()) ok = pv_step(prev);
             }
         }
     } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
         // ===================================================================== softmax + epilogue (128 threads)
         const int quad = warp & 3;                      // tensor-memory lanes this warp may touch: 32*quad .. +31
         const int row = quad * 32 + lane;               // row of the 128-row tile
         const bool lower = row >= kBlock;
         const unsigned lane_addr = tmem + ((unsigned)(quad * 32) << 16);
+        const float sl2 = p.scale_log2;
         unsigned sched_n = 0, grp_n = 0;
         bool ok = true;
+        float m_ref = -INFINITY, l_sum = 0.f;
+        bool o_dirty = false;                           // has any P V been accumulated for this tile yet
         while (ok) {
-            const unsigned ss = sched_n & 1u, sp = (sched_n >> 1) & 1u;
+            const unsigned ss = sched_n % kSchedSlots, sp = (sched_n / kSchedSlots) & 1u;
             if (!mbar_wait(&ctl->sched_full[ss], sp, ctl, p.status, 30)) break;
-            const int w = *(volatile int*)&ctl->work[ss];
+            const WorkSlot* slot = &ctl->slot[ss];
+            const int w = slot->w, flags = slot->flags, n = slot->n_steps;
+            if (w < 0) break;
+            const int my_q = lower ? slot->qb : slot->qa;
+            const bool live = flags & kSegLive;
+            if (flags & kSegFirst) {
+                m_ref = -INFINITY;
+                l_sum = 0.f;
+                o_dirty = false;
+                if (live) {
+                    // clear the accumulator (the previous tile's epilogue has already read it)
+                    tmem_st32_zero(lane_addr + kColO);
+                    tmem_st32_zero(lane_addr + kColO + 32);
+                }
+            }
+            for (int i = 0; i < n && ok; ++i) {
+                const StepEntry* e = &slot->steps[i];
+                const int full = e->full;
+                const int c0 = e->c0, c1 = e->c1;
+                const int my_c = full ? (my_q >= 0 ? c0 : -1) : (lower ? c1 : c0);          // warp-uniform
+                const int my_half = (full || !lower) ? 0 : 1;
+                ok = mbar_wait(&ctl->s_full, grp_n & 1u, ctl, p.status, 31);
+                if (!ok) break;
+                tc_fence_after();
+                float s[64];
+                if (my_c >= 0) {
+                    tmem_ld64(lane_addr + kColS + my_half * 64, s);
+                    tmem_wait_ld();
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&ctl->s_free);
+                unsigned pk[32];
+                float alpha = 1.f;
+                bool rescale = false;
+                if (my_c >= 0) {
+                    const unsigned long long kb = my_half ? e->kb1 : e->kb0;
+                    if (kb != ~0ull) {
+#pragma unroll
+                        for (int j = 0; j < 64; ++j) s[j] = ((kb >> j) & 1ull) ? s[j] : -INFINITY;
+                    }
+                    float mx0 = max3(s[0], s[1], s[2]), mx1 = max3(s[3], s[4], s[5]);
+#pragma unroll
+                    for (int j = 6; j < 62; j += 4) {
+                        mx0 = max3(mx0, s[j], s[j + 1]);
+                        mx1 = max3(mx1, s[j + 2], s[j + 3]);
+                    }
+                    const float m_cand = max3(mx0, mx1, fmaxf(s[62], s[63])) * sl2;
+                    const bool need = m_cand > m_ref + kRescaleThreshold;        // true on the first step (m_ref = -inf)
+                    rescale = __any_sync(0xffffffffu, need);
+                    if (need) {
+                        alpha = ex2(m_ref - m_cand);
+                        m_ref = m_cand;
+                    }
+                    float sum0 = 0.f, sum1 = 0.f;
+                    const float neg_m = -m_ref;
+#pragma unroll
+                    for (int j = 0; j < 64; j += 2) {
+                        float t0, t1;
+                        ffma2(t0, t1, s[j], s[j + 1], sl2, neg_m);
+                        const float p0 = ex2(t0), p1 = ex2(t1);
+                        fadd2(sum0, sum1, p0, p1);
+                        pk[j >> 1] = pack_bf16(p0, p1);
+                    }
+                    l_sum = l_sum * alpha + (sum0 + sum1);
+                }
+                // P of the previous step must have been consumed, and O must be at rest, before touching either
+                ok = mbar_wait(&ctl->pv_done, (grp_n & 1u) ^ 1u, ctl, p.status, 32);
+                if (!ok) break;
+                tc_fence_after();
+                if (rescale && o_dirty) {
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+                        float o[32];
+                        tmem_ld32(lane_addr + kColO + half * 32, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int j = 0; j < 32; j += 2) fmul2(o[j], o[j + 1], alpha);
+                        tmem_st32(lane_addr + kColO + half * 32, reinterpret_cast<unsigned*>(o));
+                    }
+                }
+                if (full) {
+                    if (my_c >= 0) tmem_st32(lane_addr + kColP, pk);
+                    else tmem_st32_zero(lane_addr + kColP);                      // tile without a lower query block
+                } else {
+                    // split step: my probabilities go to my half, zeros to the half of the other key block
+                    if (my_c >= 0) tmem_st32(lane_addr + kColP + my_half * 32, pk);
+                    const int other_c = lower ? c0 : c1;
+                    if (other_c >= 0) tmem_st32_zero(lane_addr + kColP + (lower ? 0 : 32));
+                }
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&ctl->p_full);
+                ++grp_n;
+                o_dirty = true;
+            }
+            if (!ok) break;
+            if (flags & kSegLast) {
+                // -------------------------------------------------------- epilogue of the tile
+                const int bh = slot->bh;
+                const unsigned long long qbits = lower ? slot->qbits_b : slot->qbits_a;
+                const bool have = live && o_dirty;
+                if (have) {
+                    ok = mbar_wait(&ctl->pv_done, (grp_n & 1u) ^ 1u, ctl, p.status, 33);   // last P V of the tile
+                    if (!ok) break;
+                    tc_fence_after();
+                }
+                if (my_q >= 0) {
+                    const int r64 = row & (kBlock - 1);
+                    const bool good = have && ((qbits >> r64) & 1ull) && l_sum > 0.f;
+                    const float inv = good ? 1.f / l_sum : 0.f;
+                    const size_t tok = ((size_t)bh * p.nb + my_q) * kBlock + r64;
+                    uint4* dst = reinterpret_cast<uint4*>(p.out + tok * kBlock);
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+                        float o[32];
+                        if (have) {                     // warp-uniform
+                            tmem_ld32(lane_addr + kColO + half * 32, o);
+                            tmem_wait_ld();
+                        }
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            uint4 v4;
+                            v4.x = good ? pack_bf16(o[8 * j + 0] * inv, o[8 * j + 1] * inv) : 0u;
+                            v4.y = good ? pack_bf16(o[8 * j + 2] * inv, o[8 * j + 3] * inv) : 0u;
+                            v4.z = good ? pack_bf16(o[8 * j + 4] * inv, o[8 * j + 5] * inv) : 0u;
+                            v4.w = good ? pack_bf16(o[8 * j + 6] * inv, o[8 * j + 7] * inv) : 0u;
+                            dst[half * 4 + j] = v4;
+                        }
+                    }
+                    if (p.lse) p.lse[tok] = good ? (m_ref + log2f(l_sum)) * 0.6931471805599453f : -INFINITY;
+                }
+            }
+            tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&ctl->sched_empty[ss]);
             ++sched_n;
-            if (w < 0) break;
-            const Work wk = decode_work(p, w);
-            const bool has_qb = wk.item.qb >= 0;
-            const int my_q = lower ? wk.item.qb : wk.item.qa;
-            const bool live = tile_is_live(p, wk);
-            float m_ref = -INFINITY, l_sum = 0.f;
-            bool o_dirty = false;                       // has any P V been accumulated for this tile yet
-            if (live) {
-                // clear the accumulator (the previous tile's epilogue has already read it)
-                tmem_st32_zero(lane_addr + kColO);
-                tmem_st32_zero(lane_addr + kColO + 32);
-                for (int i = 0; i < wk.item.step_count && ok; ++i) {
-                    const LiveStep l = live_step(p, wk.batch, p.steps[wk.item.step_begin + i], has_qb);
-                    if (!l.any()) continue;
-                    const int my_c = l.full ? (my_q >= 0 ? l.c0 : -1) : (lower ? l.c1 : l.c0);   // warp-uniform
-                    const int my_half = (l.full || !lower) ? 0 : 1;
-                    ok = mbar_wait(&ctl->s_full, grp_n & 1u, ctl, p.status, 31);
-                    if (!ok) break;
-                    tc_fence_after();
-                    float s[64];
-                    if (my_c >= 0) {
-                        tmem_ld64(lane_addr + kColS + my_half * 64, s);
-                        tmem_wait_ld();
-                    }
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&ctl->s_free);
-                    unsigned pk[32];
-                    float alpha = 1.f;
-                    bool rescale = false;
-                    if (my_c >= 0) {
-                        const unsigned long long kb = key_bits(p, wk.batch, my_c);
-                        if (kb != ~0ull) {
-#pragma unroll
-                            for (int j = 0; j < 64; ++j) s[j] = ((kb >> j) & 1ull) ? s[j] : -INFINITY;
-                        }
-                        float mx = s[0];
-#pragma unroll
-                        for (int j = 1; j < 64; ++j) mx = fmaxf(mx, s[j]);
-                        const float m_cand = mx * p.scale_log2;
-                        const bool need = m_cand > m_ref + kRescaleThreshold;    // true on the first step (m_ref = -inf)
-                        rescale = __any_sync(0xffffffffu, need);
-                        if (need) {
-                            alpha = ex2(m_ref - m_cand);
-                            m_ref = m_cand;
-                        }
-                        float sum = 0.f;
-#pragma unroll
-                        for (int j = 0; j < 64; j += 2) {
-                            const float p0 = ex2(fmaf(s[j], p.scale_log2, -m_ref));
-                            const float p1 = ex2(fmaf(s[j + 1], p.scale_log2, -m_ref));
-                            sum += p0 + p1;
-                            pk[j >> 1] = pack_bf16(p0, p1);
-                        }
-                        l_sum = l_sum * alpha + sum;
-                    }
-                    // P of the previous step must have been consumed, and O must be at rest, before touching either
-                    ok = mbar_wait(&ctl->pv_done, (grp_n & 1u) ^ 1u, ctl, p.status, 32);
-                    if (!ok) break;
-                    tc_fence_after();
-                    if (rescale && o_dirty) {
-                        float o[64];
-                        tmem_ld64(lane_addr + kColO, o);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int j = 0; j < 64; ++j) o[j] *= alpha;
-                        tmem_st32(lane_addr + kColO, reinterpret_cast<unsigned*>(o));
-                        tmem_st32(lane_addr + kColO + 32, reinterpret_cast<unsigned*>(o) + 32);
-                    }
-                    if (l.full) {
-                        if (my_c >= 0) tmem_st32(lane_addr + kColP, pk);
-                        else tmem_st32_zero(lane_addr + kColP);                  // tile without a lower query block
-                    } else {
-                        // split step: my probabilities go to my half, zeros to the half of the other key block
-                        if (my_c >= 0) tmem_st32(lane_addr + kColP + my_half * 32, pk);
-                        const int other_c = lower ? l.c0 : l.c1;
-                        if (other_c >= 0) tmem_st32_zero(lane_addr + kColP + (1 - (lower ? 1 : 0)) * 32);
-                    }
-                    tmem_wait_st();
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&ctl->p_full);
-                    ++grp_n;
-                    o_dirty = true;
-                }
-                if (!ok) break;
-            }
-            // ------------------------------------------------------------ epilogue of the tile
-            float o[64];
-            bool have = false;
-            if (live && o_dirty) {
-                ok = mbar_wait(&ctl->pv_done, (grp_n & 1u) ^ 1u, ctl, p.status, 33);   // last P V of the tile
-                if (!ok) break;
-                tc_fence_after();
-                tmem_ld64(lane_addr + kColO, o);
-                tmem_wait_ld();
-                have = true;
-            }
-            if (my_q >= 0) {
-                const int r64 = row & (kBlock - 1);
-                const bool q_valid = (key_bits(p, wk.batch, my_q) >> r64) & 1ull;
-                const bool good = have && q_valid && l_sum > 0.f;
-                const float inv = good ? 1.f / l_sum : 0.f;
-                const size_t tok = ((size_t)wk.bh * p.nb + my_q) * kBlock + r64;
-                uint4* dst = reinterpret_cast<uint4*>(p.out + tok * kBlock);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    uint4 v4;
-                    v4.x = good ? pack_bf16(o[8 * j + 0] * inv, o[8 * j + 1] * inv) : 0u;
-                    v4.y = good ? pack_bf16(o[8 * j + 2] * inv, o[8 * j + 3] * inv) : 0u;
-                    v4.z = good ? pack_bf16(o[8 * j + 4] * inv, o[8 * j + 5] * inv) : 0u;
-                    v4.w = good ? pack_bf16(o[8 * j + 6] * inv, o[8 * j + 7] * inv) : 0u;
-                    dst[j] = v4;
-                }
-                if (p.lse) p.lse[tok] = good ? (m_ref + log2f(l_sum)) * 0.6931471805599453f : -INFINITY;
-            }
         }
     }
 
