@@ -82,14 +82,15 @@ BIGBIRD_API int bigbird_layout_export(const bigbird_layout* layout, int32_t* row
 
 /*
  * Introspection of the tile schedule derived from the lists (used by the tests; not needed to run attention).
- * The tensor-core kernel stacks two query blocks into one 2b-row tile and walks a list of steps: a full step
- * is one key block attended by both halves of the tile, a split step pairs a key block attended only by the
- * upper half with one attended only by the lower half.
+ * The tensor-core kernel stacks two query blocks into one 2b-row tile (upper half, lower half) and walks a
+ * list of steps; a step is one key block together with the halves of the tile that attend it.
  *   sizes   host int32[4]: items per head, leading "heavy" (global-tile) items per head, total steps, heads
  *   items   host int32[H * items_per_head * 8] or NULL: per item (qa, qb, step_begin, step_count, part, nparts, tile, 0),
- *           step_begin relative to the head's first step
+ *           qa / qb the query blocks of the upper / lower half (qb == -1: none), step_begin relative to the
+ *           head's first step
  *   step_base host int32[H] or NULL: first step of each head
- *   steps   host int32[total_steps * 2] or NULL: (c0, c1); c1 == -2 marks a full step, -1 marks "no block"
+ *   steps   host int32[total_steps * 2] or NULL: (key block, who) with who = 0 both halves, 1 upper half only,
+ *           2 lower half only
  */
 BIGBIRD_API int bigbird_layout_schedule(const bigbird_layout* layout, int32_t* sizes, int32_t* items, int32_t* step_base,
                             int32_t* steps);

@@ -3,16 +3,21 @@
 // What is computed: Eq. (AT) of arXiv 2007.14062 (softmax attention restricted to the out-neighbours of each
 // query) over the block graph of App. D.  How, on B200:
 //
-//   * Two query blocks are stacked into one 128-row tile so that every tcgen05.mma runs at M = 128.  The
-//     tile walks a list of steps prepared on the host: a full step is a key block both halves attend; a split
-//     step pairs a key block only the upper half attends with one only the lower half attends.
-//   * A producer warp fetches Q once per tile and the K and V blocks of each step with TMA (128-byte swizzle)
-//     straight from the [B, H, N, D] tensors into a shared-memory ring: nothing is gathered or packed in HBM.
-//   * One thread issues S = Q K^T and O += P V as tcgen05.mma (bf16 operands, fp32 accumulators in tensor
-//     memory).  P is handed to the second MMA through tensor memory.
-//   * Four softmax warps own one row each per thread: tcgen05.ld of the scores, key-padding mask, running
-//     maximum and sum in fp32 (base-2 exponentials), bf16 probabilities written back with tcgen05.st.  The
-//     accumulator is rescaled only when the running maximum grows by more than 2^8.
+//   * Two query blocks are stacked into one 128-row tile so that every tcgen05.mma runs at M = 128.  The tile
+//     walks a list of key blocks prepared on the host; each is attended by both halves of the tile or by one.
+//     The MMAs always cover all 128 rows; rows that do not attend a key block get probability zero for it.
+//   * A producer thread fetches Q once per tile and the K and V blocks with TMA (128-byte swizzle) straight
+//     from the [B, H, N, D] tensors into a shared-memory ring: nothing is gathered or packed in HBM.
+//   * Key blocks are processed three at a time (one "step").  Their K tiles land in three adjacent ring slots, so
+//     that S = Q K^T of a step is one N = 192 tcgen05.mma per 16 head dimensions (an MMA instruction costs its
+//     issuing thread about the same time whatever its N, so wide MMAs are the cheap ones).  O += P V follows
+//     with P read from tensor memory, where the bf16 probabilities of a block overwrite its own scores.
+//   * Eight softmax warps: two threads share a row, each owning 32 of the 64 score columns of a key block.
+//     Pass 1 finds the row maximum (the two threads exchange theirs through shared memory), pass 2 re-reads
+//     the scores, applies the key-padding mask, exponentiates (base 2, fp32), sums, and writes the
+//     probabilities back.  The accumulator is rescaled only when the running maximum grows by more than 2^8.
+//     The two partial row sums meet at the end of the tile.  The output of a tile is written while the first
+//     step of the next tile is already in flight.
 //   * CTAs are persistent and draw work from a global counter: global-row tiles first, then the sparse tiles
 //     in (batch, head)-major order.  Two CTAs share an SM so that one's softmax overlaps the other's MMAs.
 //
@@ -32,55 +37,54 @@ namespace {
 // ------------------------------------------------------------------------------------------------ constants
 constexpr int kBlock = 64;                 // tokens per block (b) and head dimension (D)
 constexpr int kTileBytes = kBlock * kBlock * 2;      // one 64x64 bf16 tile
-constexpr int kRingSlots = 10;
-constexpr int kThreads = 256;              // warp 0 TMA, warp 1 MMA issuer, warp 2 scheduler, warp 3 idle, warps 4..7 softmax
-constexpr int kSoftmaxWarps = 4;
-#ifndef BB_REGS_LIGHT
-#define BB_REGS_LIGHT 64
-#define BB_REGS_SOFTMAX 192
-#endif
-constexpr int kRegsLight = BB_REGS_LIGHT;             // registers per thread of warps 0..3 after setmaxnreg
-constexpr int kRegsSoftmax = BB_REGS_SOFTMAX;          // registers per thread of warps 4..7 after setmaxnreg
+constexpr int kStepChunks = 3;             // key blocks per step
+constexpr int kRingGroups = 3;             // ring of groups of kStepChunks adjacent tiles (the K or the V blocks of one step)
+constexpr int kGroupBytes = kStepChunks * kTileBytes;
+constexpr int kThreads = 384;              // warp 0 TMA, warp 1 MMA issuer, warp 2 scheduler, warp 3 idle, warps 4..11 softmax
+constexpr int kSoftmaxWarps = 8;
 constexpr int kTmemCols = 256;
-constexpr int kColS = 0;                   // scores: 2 x 64 fp32 columns
-constexpr int kColP = 128;                 // probabilities: 2 x 32 columns of packed bf16 pairs
-constexpr int kColO = 192;                 // output accumulator: 64 fp32 columns
+constexpr int kColS = 0;                   // kStepChunks x 64 fp32 score columns; a block's probabilities reuse its columns
+constexpr int kColO = kStepChunks * 64;    // output accumulator: 64 fp32 columns
 constexpr float kRescaleThreshold = 8.0f;  // in log2 units
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+constexpr long long kWaitLimitCycles = 4000000000ll;   // about two seconds
 constexpr int kSchedSlots = 3;
-constexpr int kSegSteps = 64;              // live steps per posted segment of a tile
+constexpr int kSegChunks = 96;             // live key blocks per posted segment of a tile (a multiple of kStepChunks)
+static_assert(kColO + 64 <= kTmemCols && kSegChunks % kStepChunks == 0, "tensor-memory and segment layout");
 
-// A step of a tile after the key-padding mask has been applied: key blocks that are entirely padding are gone.
-struct __align__(16) StepEntry {
-    int c0, c1;                    // key block of the upper / lower half (or of both when full), -1 = none
-    int full;
-    int pad_;
-    unsigned long long kb0, kb1;   // valid-key bits of c0 / c1
+// A key block of a tile after the key-padding mask has been applied.
+struct __align__(16) ChunkEntry {
+    int c;                         // key block
+    int who;                       // kBothHalves, kUpperHalf or kLowerHalf: the halves of the tile that attend it
+    unsigned long long kb;         // valid-key bits (never 0: blocks that are entirely padding are dropped)
 };
 enum { kSegFirst = 1, kSegLast = 2, kSegLive = 4 };
 struct __align__(16) WorkSlot {
     int w;                         // work index, -1 = no more work
     int bh, batch, qa, qb;
-    int n_steps;
+    int n_chunks;
     int flags;
     int pad_;
     unsigned long long qbits_a, qbits_b;
-    StepEntry steps[kSegSteps];
+    ChunkEntry chunks[kSegChunks];
 };
 
 struct __align__(16) SmemCtl {
-    unsigned long long full[kRingSlots];
-    unsigned long long empty[kRingSlots];
+    unsigned long long full[kRingGroups];
+    unsigned long long empty[kRingGroups];
     unsigned long long q_full, q_empty;
-    unsigned long long s_full, s_free, p_full, pv_done;
+    unsigned long long s_full, p_full;
+    unsigned long long x_ready[4];         // per 32-row group: both column halves have posted their row maxima
+    unsigned long long l_ready[4];         // per 32-row group: both column halves have posted their row sums
     unsigned long long sched_full[kSchedSlots], sched_empty[kSchedSlots];
+    float x_part[2][2][128];               // [step parity][column half][row]
+    float l_part[2][2][128];               // [tile parity][column half][row]
     unsigned tmem_base;
     int abort_flag;
     WorkSlot slot[kSchedSlots];
 };
 constexpr int kSmemQ = 0;
 constexpr int kSmemRing = 2 * kTileBytes;
-constexpr int kSmemCtl = kSmemRing + kRingSlots * kTileBytes;
+constexpr int kSmemCtl = kSmemRing + kRingGroups * kGroupBytes;
 constexpr int kSmemBytes = kSmemCtl + (int)sizeof(SmemCtl) + 1024;   // + slack for the 1024-byte alignment
 
 struct KernelParams {
@@ -124,14 +128,18 @@ __device__ __forceinline__ unsigned long long global_ns() {
     return t;
 }
 
-// Bounded wait.  Returns false if the wait expired or another thread of the CTA already gave up.
+// Bounded wait.  Returns false if the wait expired or another thread of the CTA already gave up.  The limit is
+// counted in SM clock cycles (a read of the cycle counter is cheap, unlike one of the global nanosecond timer)
+// and the counter is first read only after 64 failed tries.
 __device__ __forceinline__ bool mbar_wait_slow(unsigned long long* bar, unsigned parity, SmemCtl* ctl, int* status, int code) {
-    const unsigned long long t0 = global_ns();
+    long long t0 = 0;
     for (unsigned it = 0;; ++it) {
         if (mbar_try(bar, parity)) return true;
         if ((it & 63u) == 63u) {
             if (*(volatile int*)&ctl->abort_flag) return false;
-            if (global_ns() - t0 > kWaitLimitNs) {
+            const long long now = clock64();
+            if (it == 63u) t0 = now;
+            if (now - t0 > kWaitLimitCycles) {
                 if (atomicCAS(status, 0, BIGBIRD_ETIMEOUT) == 0) status[1] = code;
                 *(volatile int*)&ctl->abort_flag = 1;
                 return false;
@@ -178,25 +186,15 @@ __device__ __forceinline__ unsigned long long smem_desc_sw128(unsigned addr) {
          | (1ull << 46)                       // descriptor version of sm_100
          | (2ull << 61);                      // SWIZZLE_128B
 }
-// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 64; B is K-major (K^T) or MN-major (V).
-constexpr unsigned kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
-constexpr unsigned kIdescPV = kIdescQK | (1u << 16);
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 64 (Q K^T adds 64 per further key block); B is K-major (K^T) or MN-major (V).
+constexpr unsigned kIdescQK64 = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);   // N field (bits 17..22) = N / 8
+constexpr unsigned kIdescPV = kIdescQK64 | (1u << 16);
 
 #define BB_REP32(F, o) F(o+0), F(o+1), F(o+2), F(o+3), F(o+4), F(o+5), F(o+6), F(o+7), F(o+8), F(o+9), F(o+10), F(o+11), \
     F(o+12), F(o+13), F(o+14), F(o+15), F(o+16), F(o+17), F(o+18), F(o+19), F(o+20), F(o+21), F(o+22), F(o+23), \
     F(o+24), F(o+25), F(o+26), F(o+27), F(o+28), F(o+29), F(o+30), F(o+31)
 #define BB_OUT(i) "=r"(u[i])
 #define BB_IN(i) "r"(u[i])
-__device__ __forceinline__ void tmem_ld64(unsigned taddr, float* r) {
-    unsigned* u = reinterpret_cast<unsigned*>(r);
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x64.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, "
-        "%32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, "
-        "%48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];"
-        : BB_REP32(BB_OUT, 0), BB_REP32(BB_OUT, 32) : "r"(taddr) : "memory");
-}
 __device__ __forceinline__ void tmem_ld32(unsigned taddr, float* r) {
     unsigned* u = reinterpret_cast<unsigned*>(r);
     asm volatile(
@@ -212,14 +210,28 @@ __device__ __forceinline__ void tmem_st32(unsigned taddr, const unsigned* u) {
         "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31};"
         ::BB_REP32(BB_IN, 0), "r"(taddr) : "memory");
 }
+#define BB_REP16(F, o) F(o+0), F(o+1), F(o+2), F(o+3), F(o+4), F(o+5), F(o+6), F(o+7), F(o+8), F(o+9), F(o+10), F(o+11), \
+    F(o+12), F(o+13), F(o+14), F(o+15)
+__device__ __forceinline__ void tmem_ld16(unsigned taddr, float* r) {
+    unsigned* u = reinterpret_cast<unsigned*>(r);
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : BB_REP16(BB_OUT, 0) : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st16(unsigned taddr, const unsigned* u) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15};"
+        ::BB_REP16(BB_IN, 0), "r"(taddr) : "memory");
+}
 #undef BB_OUT
 #undef BB_IN
-__device__ __forceinline__ void tmem_st32_zero(unsigned taddr) {
+__device__ __forceinline__ void tmem_st16_zero(unsigned taddr) {
     const unsigned z = 0;
     asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%1], "
-        "{%0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, "
-        "%0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0};"
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%1], "
+        "{%0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0};"
         ::"r"(z), "r"(taddr) : "memory");
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
@@ -260,6 +272,15 @@ __device__ __forceinline__ unsigned long long key_bits(const KernelParams& p, in
     if (c < 0) return 0ull;
     return p.kbits ? p.kbits[(size_t)batch * p.nb + c] : ~0ull;
 }
+__device__ __forceinline__ float row_max32(const float* s) {
+    float mx0 = max3(s[0], s[1], s[2]), mx1 = max3(s[3], s[4], s[5]);
+#pragma unroll
+    for (int j = 6; j < 30; j += 4) {
+        mx0 = max3(mx0, s[j], s[j + 1]);
+        mx1 = max3(mx1, s[j + 2], s[j + 3]);
+    }
+    return max3(mx0, mx1, fmaxf(s[30], s[31]));
+}
 
 // ------------------------------------------------------------------------------------------------ the kernel
 __global__ void __launch_bounds__(kThreads, 2)
@@ -271,13 +292,12 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < kRingSlots; ++i) { mbar_init(&ctl->full[i], 1); mbar_init(&ctl->empty[i], 1); }
+        for (int i = 0; i < kRingGroups; ++i) { mbar_init(&ctl->full[i], 1); mbar_init(&ctl->empty[i], 1); }
         mbar_init(&ctl->q_full, 1);
         mbar_init(&ctl->q_empty, 1);
         mbar_init(&ctl->s_full, 1);
-        mbar_init(&ctl->s_free, kSoftmaxWarps);
         mbar_init(&ctl->p_full, kSoftmaxWarps);
-        mbar_init(&ctl->pv_done, 1);
+        for (int i = 0; i < 4; ++i) { mbar_init(&ctl->x_ready[i], 2); mbar_init(&ctl->l_ready[i], 2); }
         for (int i = 0; i < kSchedSlots; ++i) { mbar_init(&ctl->sched_full[i], 1); mbar_init(&ctl->sched_empty[i], 2 + kSoftmaxWarps); }
         ctl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -293,9 +313,8 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     const unsigned tmem = *(volatile unsigned*)&ctl->tmem_base;
 
     if (warp < 4) {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsLight));
         if (warp == 2) {
-            // ================================================================= scheduler: fetch work, post live steps
+            // ================================================================= scheduler: fetch work, post live key blocks
             unsigned sched_n = 0;
             bool ok = true;
             const unsigned lt_mask = (1u << lane) - 1u;
@@ -321,7 +340,6 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                     item = p.items[(size_t)(bh % p.H) * p.items_per_head + it];
                 }
                 const int batch = bh / p.H;
-                const bool has_qb = item.qb >= 0;
                 const unsigned long long qbits_a = w >= 0 ? key_bits(p, batch, item.qa) : 0ull;
                 const unsigned long long qbits_b = w >= 0 ? key_bits(p, batch, item.qb) : 0ull;
                 const bool tile_live = (qbits_a | qbits_b) != 0ull;      // a tile whose query rows are all padding is skipped
@@ -334,20 +352,22 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                     if (!ok) break;
                     WorkSlot* slot = &ctl->slot[ss];
                     int count = 0;
-                    while (i0 < n_raw && count <= kSegSteps - 32) {
+                    while (i0 < n_raw && count <= kSegChunks - 32) {
                         const int i = i0 + lane;
-                        StepEntry e{-1, -1, 0, 0, 0ull, 0ull};
+                        ChunkEntry e{-1, 0, 0ull};
+                        bool alive = false;
                         if (i < n_raw) {
                             const Step s = p.steps[item.step_begin + i];
-                            e.full = s.c1 == kStepFull;
-                            e.kb0 = key_bits(p, batch, s.c0);
-                            e.kb1 = (!e.full && has_qb) ? key_bits(p, batch, s.c1) : 0ull;
-                            e.c0 = e.kb0 ? s.c0 : -1;
-                            e.c1 = e.kb1 ? s.c1 : -1;
+                            // halves whose query rows are all padding do not attend anything
+                            const bool ua = s.who != kLowerHalf && qbits_a != 0ull;
+                            const bool ub = s.who != kUpperHalf && qbits_b != 0ull;
+                            e.c = s.c;
+                            e.who = (ua && ub) ? kBothHalves : (ua ? kUpperHalf : kLowerHalf);
+                            e.kb = key_bits(p, batch, s.c);
+                            alive = e.kb != 0ull && (ua || ub);
                         }
-                        const bool alive = e.c0 >= 0 || e.c1 >= 0;
                         const unsigned bal = __ballot_sync(0xffffffffu, alive);
-                        if (alive) slot->steps[count + __popc(bal & lt_mask)] = e;
+                        if (alive) slot->chunks[count + __popc(bal & lt_mask)] = e;
                         count += __popc(bal);
                         i0 += 32;
                     }
@@ -357,7 +377,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                         slot->batch = batch;
                         slot->qa = item.qa;
                         slot->qb = item.qb;
-                        slot->n_steps = count;
+                        slot->n_chunks = count;
                         slot->flags = (first ? kSegFirst : 0) | (i0 >= n_raw ? kSegLast : 0) | (tile_live ? kSegLive : 0);
                         slot->qbits_a = qbits_a;
                         slot->qbits_b = qbits_b;
@@ -372,27 +392,26 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             }
         } else if (warp == 0 && lane == 0) {
             // ================================================================= TMA producer
+            // Ring order = the order in which the MMA thread consumes groups: V of step i-1, then K of step i.
             unsigned ring_n = 0, q_n = 0, sched_n = 0;
             bool ok = true;
-            auto load = [&](const CUtensorMap* tm, int bh, int block) -> bool {
-                const unsigned slot = ring_n % kRingSlots, ph = (ring_n / kRingSlots) & 1u;
-                if (!mbar_wait(&ctl->empty[slot], ph ^ 1u, ctl, p.status, 10)) return false;
-                mbar_expect_tx(&ctl->full[slot], kTileBytes);
-                tma_load_tile(smem + kSmemRing + slot * kTileBytes, tm, (bh * p.nb + block) * kBlock, &ctl->full[slot]);
+            // the (up to three) blocks c[0..cnt) of K or V into the next group of adjacent ring slots
+            auto load_group = [&](const CUtensorMap* tm, int bh, const int* c, int cnt) -> bool {
+                const unsigned g = ring_n % kRingGroups, ph = (ring_n / kRingGroups) & 1u;
+                if (!mbar_wait(&ctl->empty[g], ph ^ 1u, ctl, p.status, 10)) return false;
+                mbar_expect_tx(&ctl->full[g], cnt * kTileBytes);
+#pragma unroll
+                for (int j = 0; j < kStepChunks; ++j)
+                    if (j < cnt) tma_load_tile(smem + kSmemRing + g * kGroupBytes + j * kTileBytes, tm, (bh * p.nb + c[j]) * kBlock, &ctl->full[g]);
                 ++ring_n;
                 return true;
             };
-            auto load_pair = [&](const CUtensorMap* tm, int bh, int c0, int c1) -> bool {
-                if (c0 >= 0 && !load(tm, bh, c0)) return false;
-                if (c1 >= 0 && !load(tm, bh, c1)) return false;
-                return true;
-            };
-            int prev_c0 = -1, prev_c1 = -1;
+            int pend_n = 0, pend_bh = 0, pend_c[kStepChunks] = {0, 0, 0};
             while (ok) {
                 const unsigned ss = sched_n % kSchedSlots, sp = (sched_n / kSchedSlots) & 1u;
                 if (!mbar_wait(&ctl->sched_full[ss], sp, ctl, p.status, 13)) break;
                 const WorkSlot* slot = &ctl->slot[ss];
-                const int w = slot->w, flags = slot->flags, bh = slot->bh, n = slot->n_steps;
+                const int w = slot->w, flags = slot->flags, bh = slot->bh, n = slot->n_chunks;
                 if (w >= 0 && (flags & kSegLive)) {
                     if (flags & kSegFirst) {
                         const int qa = slot->qa, qb = slot->qb;
@@ -402,205 +421,247 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                         tma_load_tile(smem + kSmemQ, &tm_q, (bh * p.nb + qa) * kBlock, &ctl->q_full);
                         if (qb >= 0) tma_load_tile(smem + kSmemQ + kTileBytes, &tm_q, (bh * p.nb + qb) * kBlock, &ctl->q_full);
                         ++q_n;
-                        prev_c0 = prev_c1 = -1;
                     }
-                    // K of step i+1 goes ahead of V of step i: the order in which the MMA thread consumes them
-                    for (int i = 0; i < n && ok; ++i) {
-                        const int c0 = slot->steps[i].c0, c1 = slot->steps[i].c1;
-                        ok = load_pair(&tm_k, bh, c0, c1);
-                        if (ok) ok = load_pair(&tm_v, bh, prev_c0, prev_c1);
-                        prev_c0 = c0;
-                        prev_c1 = c1;
+                    for (int i = 0; i < n && ok; i += kStepChunks) {
+                        if (pend_n > 0) ok = load_group(&tm_v, pend_bh, pend_c, pend_n);
+                        if (!ok) break;
+                        pend_n = min(kStepChunks, n - i);
+#pragma unroll
+                        for (int j = 0; j < kStepChunks; ++j)
+                            if (j < pend_n) pend_c[j] = slot->chunks[i + j].c;
+                        pend_bh = bh;
+                        ok = load_group(&tm_k, bh, pend_c, pend_n);
                     }
-                    if (ok && (flags & kSegLast)) ok = load_pair(&tm_v, bh, prev_c0, prev_c1);
                 }
                 mbar_arrive(&ctl->sched_empty[ss]);
                 ++sched_n;
-                if (w < 0) break;
+                if (w < 0) {
+                    if (ok && pend_n > 0) load_group(&tm_v, pend_bh, pend_c, pend_n);
+                    break;
+                }
             }
         } else if (warp == 1 && lane == 0) {
             // ================================================================= MMA issuer
-            unsigned ring_n = 0, q_n = 0, sched_n = 0, grp_n = 0, pv_n = 0;   // grp_n: live steps whose Q K^T was issued
+            unsigned ring_n = 0, q_n = 0, sched_n = 0, pv_n = 0;
             bool ok = true;
             const unsigned long long q_desc = smem_desc_sw128(smem_u32(smem + kSmemQ));
-            auto qk = [&](int col_off) -> bool {        // S[:, col_off .. col_off+63] = Q K^T with K in the next ring slot
-                const unsigned slot = ring_n % kRingSlots, ph = (ring_n / kRingSlots) & 1u;
-                if (!mbar_wait(&ctl->full[slot], ph, ctl, p.status, 20)) return false;
+            auto qk = [&](int cnt) -> bool {            // S[:, 0 .. 64 cnt) = Q K^T with the K blocks of the next ring group
+                const unsigned g = ring_n % kRingGroups, ph = (ring_n / kRingGroups) & 1u;
+                if (!mbar_wait(&ctl->full[g], ph, ctl, p.status, 20)) return false;
                 tc_fence_after();
-                const unsigned long long k_desc = smem_desc_sw128(smem_u32(smem + kSmemRing + slot * kTileBytes));
+                // the blocks of a group are adjacent: their 64 cnt rows form one K-major operand
+                const unsigned long long k_desc = smem_desc_sw128(smem_u32(smem + kSmemRing + g * kGroupBytes));
+                const unsigned idesc = kIdescQK64 + ((unsigned)(cnt - 1) << 20);           // N = 64 cnt
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk)          // 16 head dims (32 bytes inside the swizzled row) per MMA
-                    mma_ss(tmem + kColS + col_off, q_desc + (unsigned long long)(kk * 2), k_desc + (unsigned long long)(kk * 2), kIdescQK, kk > 0);
-                tc_commit(&ctl->empty[slot]);
+                    mma_ss(tmem + kColS, q_desc + (unsigned long long)(kk * 2), k_desc + (unsigned long long)(kk * 2), idesc, kk > 0);
+                tc_commit(&ctl->empty[g]);
                 ++ring_n;
                 return true;
             };
-            auto pv = [&](int p_col_off) -> bool {      // O += P[:, 64 keys] V with V in the next ring slot
-                const unsigned slot = ring_n % kRingSlots, ph = (ring_n / kRingSlots) & 1u;
-                if (!mbar_wait(&ctl->full[slot], ph, ctl, p.status, 21)) return false;
-                tc_fence_after();
-                const unsigned long long v_desc = smem_desc_sw128(smem_u32(smem + kSmemRing + slot * kTileBytes));
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk)          // 16 keys per MMA: 8 packed columns of P, two 8-row groups of V
-                    mma_ts(tmem + kColO, tmem + kColP + p_col_off + kk * 8, v_desc + (unsigned long long)(kk * (2048 >> 4)), kIdescPV, 1u);
-                tc_commit(&ctl->empty[slot]);
-                ++ring_n;
-                return true;
-            };
-            auto pv_step = [&](int c0, int c1) -> bool {
+            bool pend_fresh = false;                    // the pending P V is the first of its tile: it overwrites O
+            int pend_n = 0;
+            auto pending_pv = [&]() -> bool {           // O (+)= sum_j P_j V_j with the V blocks of the next ring group
+                if (pend_n == 0) return true;
                 if (!mbar_wait(&ctl->p_full, pv_n & 1u, ctl, p.status, 22)) return false;
+                const unsigned g = ring_n % kRingGroups, ph = (ring_n / kRingGroups) & 1u;
+                if (!mbar_wait(&ctl->full[g], ph, ctl, p.status, 21)) return false;
                 tc_fence_after();
-                if (c0 >= 0 && !pv(0)) return false;
-                if (c1 >= 0 && !pv(32)) return false;
-                tc_commit(&ctl->pv_done);
+                const unsigned long long v_desc = smem_desc_sw128(smem_u32(smem + kSmemRing + g * kGroupBytes));
+#pragma unroll
+                for (int j = 0; j < kStepChunks; ++j) {
+                    if (j < pend_n) {
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk) {
+                            // 16 keys per MMA.  Keys 0..31 of a block sit in packed columns 0..15 of its score columns,
+                            // keys 32..63 in columns 32..47 (each softmax thread writes inside its own score columns).
+                            const unsigned a_col = kColS + 64 * j + (kk >> 1) * 32 + (kk & 1) * 8;
+                            mma_ts(tmem + kColO, tmem + a_col, v_desc + (unsigned long long)((j * kTileBytes + kk * 2048) >> 4), kIdescPV,
+                                   (j > 0 || kk > 0 || !pend_fresh) ? 1u : 0u);
+                        }
+                    }
+                }
+                tc_commit(&ctl->empty[g]);
+                ++ring_n;
                 ++pv_n;
+                pend_n = 0;
+                pend_fresh = false;
                 return true;
             };
-            int prev_c0 = -1, prev_c1 = -1;
             while (ok) {
                 const unsigned ss = sched_n % kSchedSlots, sp = (sched_n / kSchedSlots) & 1u;
                 if (!mbar_wait(&ctl->sched_full[ss], sp, ctl, p.status, 23)) break;
                 const WorkSlot* slot = &ctl->slot[ss];
-                const int w = slot->w, flags = slot->flags, n = slot->n_steps;
+                const int w = slot->w, flags = slot->flags, n = slot->n_chunks;
                 if (w >= 0 && (flags & kSegLive)) {
-                    if (flags & kSegFirst) {
-                        ok = mbar_wait(&ctl->q_full, q_n & 1u, ctl, p.status, 24);
+                    bool first = flags & kSegFirst;
+                    for (int i = 0; i < n && ok; i += kStepChunks) {
+                        // P V of the previous step first: the scores of this step overwrite its probabilities,
+                        // and MMAs execute in issue order
+                        ok = pending_pv();
                         if (!ok) break;
-                        tc_fence_after();
-                        prev_c0 = prev_c1 = -1;
-                    }
-                    for (int i = 0; i < n && ok; ++i) {
-                        const int c0 = slot->steps[i].c0, c1 = slot->steps[i].c1;
-                        // the softmax warps must have pulled the previous scores out of tensor memory
-                        ok = mbar_wait(&ctl->s_free, (grp_n & 1u) ^ 1u, ctl, p.status, 25);
+                        if (first) {
+                            ok = mbar_wait(&ctl->q_full, q_n & 1u, ctl, p.status, 24);
+                            if (!ok) break;
+                            tc_fence_after();
+                        }
+                        const int cnt = min(kStepChunks, n - i);
+                        ok = qk(cnt);
                         if (!ok) break;
-                        tc_fence_after();
-                        if (c0 >= 0) ok = qk(0);
-                        if (ok && c1 >= 0) ok = qk(64);
-                        if (!ok) break;
-                        tc_commit(&ctl->s_full);
-                        ++grp_n;
-                        if (prev_c0 >= 0 || prev_c1 >= 0) ok = pv_step(prev_c0, prev_c1);
-                        prev_c0 = c0;
-                        prev_c1 = c1;
+                        tc_commit(&ctl->s_full);        // also says: every earlier P V has completed
+                        pend_n = cnt;
+                        pend_fresh = first;
+                        first = false;
                     }
                     if (!ok) break;
                     if (flags & kSegLast) {
                         tc_commit(&ctl->q_empty);       // every Q K^T of the tile has been issued
                         ++q_n;
-                        if (prev_c0 >= 0 || prev_c1 >= 0) ok = pv_step(prev_c0, prev_c1);
                     }
                 }
                 mbar_arrive(&ctl->sched_empty[ss]);
                 ++sched_n;
-                if (w < 0) break;
+                if (w < 0) {
+                    if (pend_n > 0 && pending_pv()) tc_commit(&ctl->s_full);   // the last tile's accumulator is complete
+                    break;
+                }
             }
         }
     } else {
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
-        // ===================================================================== softmax + epilogue (128 threads)
+        // ===================================================================== softmax + epilogue (256 threads)
         const int quad = warp & 3;                      // tensor-memory lanes this warp may touch: 32*quad .. +31
+        const int chalf = (warp - 4) >> 2;              // which 32 of a key block's 64 score columns this thread owns
         const int row = quad * 32 + lane;               // row of the 128-row tile
         const bool lower = row >= kBlock;
+        const int my_who = lower ? kLowerHalf : kUpperHalf;
         const unsigned lane_addr = tmem + ((unsigned)(quad * 32) << 16);
+        const unsigned my_col = kColS + chalf * 32;     // first of my score columns in key block 0 of a step
         const float sl2 = p.scale_log2;
-        unsigned sched_n = 0, grp_n = 0;
+        unsigned sched_n = 0, grp_n = 0, x_n = 0, epi_n = 0;
         bool ok = true;
-        float m_ref = -INFINITY, l_sum = 0.f;
-        bool o_dirty = false;                           // has any P V been accumulated for this tile yet
+        float m_ref = -INFINITY, l_sum = 0.f;           // l_sum: this thread's columns only
+        bool o_dirty = false;                           // has any P V been issued for this tile yet
+        // output of the previous tile, written once its last P V is known to be complete
+        bool pend_out = false, pend_good = false;
+        float pend_inv = 0.f;
+        uint4* pend_dst = nullptr;
+        auto write_out = [&]() {                        // this thread's 32 accumulator columns of its row
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                float o[16];
+                tmem_ld16(lane_addr + kColO + chalf * 32 + c * 16, o);
+                tmem_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    uint4 v4;
+                    v4.x = pend_good ? pack_bf16(o[8 * j + 0] * pend_inv, o[8 * j + 1] * pend_inv) : 0u;
+                    v4.y = pend_good ? pack_bf16(o[8 * j + 2] * pend_inv, o[8 * j + 3] * pend_inv) : 0u;
+                    v4.z = pend_good ? pack_bf16(o[8 * j + 4] * pend_inv, o[8 * j + 5] * pend_inv) : 0u;
+                    v4.w = pend_good ? pack_bf16(o[8 * j + 6] * pend_inv, o[8 * j + 7] * pend_inv) : 0u;
+                    pend_dst[2 * c + j] = v4;
+                }
+            }
+            pend_out = false;
+        };
         while (ok) {
             const unsigned ss = sched_n % kSchedSlots, sp = (sched_n / kSchedSlots) & 1u;
             if (!mbar_wait(&ctl->sched_full[ss], sp, ctl, p.status, 30)) break;
             const WorkSlot* slot = &ctl->slot[ss];
-            const int w = slot->w, flags = slot->flags, n = slot->n_steps;
-            if (w < 0) break;
-            const int my_q = lower ? slot->qb : slot->qa;
+            const int w = slot->w, flags = slot->flags, n = slot->n_chunks;
+            if (w < 0) {
+                if (pend_out) {                         // warp-uniform
+                    ok = mbar_wait(&ctl->s_full, grp_n & 1u, ctl, p.status, 35);
+                    if (!ok) break;
+                    tc_fence_after();
+                    write_out();
+                }
+                break;
+            }
             const bool live = flags & kSegLive;
             if (flags & kSegFirst) {
                 m_ref = -INFINITY;
                 l_sum = 0.f;
                 o_dirty = false;
-                if (live) {
-                    // clear the accumulator (the previous tile's epilogue has already read it)
-                    tmem_st32_zero(lane_addr + kColO);
-                    tmem_st32_zero(lane_addr + kColO + 32);
-                }
             }
-            for (int i = 0; i < n && ok; ++i) {
-                const StepEntry* e = &slot->steps[i];
-                const int full = e->full;
-                const int c0 = e->c0, c1 = e->c1;
-                const int my_c = full ? (my_q >= 0 ? c0 : -1) : (lower ? c1 : c0);          // warp-uniform
-                const int my_half = (full || !lower) ? 0 : 1;
+            for (int i = 0; i < n && ok; i += kStepChunks) {
+                const ChunkEntry* e = &slot->chunks[i];
+                const int cnt = min(kStepChunks, n - i);
                 ok = mbar_wait(&ctl->s_full, grp_n & 1u, ctl, p.status, 31);
                 if (!ok) break;
                 tc_fence_after();
-                float s[64];
-                if (my_c >= 0) {
-                    tmem_ld64(lane_addr + kColS + my_half * 64, s);
+                // every P V issued before this step's scores has completed: the accumulator is at rest
+                if (pend_out) write_out();              // warp-uniform
+                // ---- pass 1: maximum of my columns over the key blocks my half of the tile attends
+                float s[32];
+                float m_loc = -INFINITY;
+                bool any_mine = false;
+#pragma unroll 1
+                for (int j = 0; j < cnt; ++j) {
+                    const int who = e[j].who;
+                    if (who != kBothHalves && who != my_who) continue;                      // warp-uniform
+                    any_mine = true;
+                    tmem_ld32(lane_addr + my_col + 64 * j, s);
                     tmem_wait_ld();
+                    const unsigned kbo = (unsigned)(e[j].kb >> (chalf * 32));
+                    if (kbo != ~0u) {
+#pragma unroll
+                        for (int t = 0; t < 32; ++t) s[t] = ((kbo >> t) & 1u) ? s[t] : -INFINITY;
+                    }
+                    m_loc = fmaxf(m_loc, row_max32(s));
                 }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&ctl->s_free);
-                unsigned pk[32];
                 float alpha = 1.f;
-                bool rescale = false;
-                if (my_c >= 0) {
-                    const unsigned long long kb = my_half ? e->kb1 : e->kb0;
-                    if (kb != ~0ull) {
-#pragma unroll
-                        for (int j = 0; j < 64; ++j) s[j] = ((kb >> j) & 1ull) ? s[j] : -INFINITY;
-                    }
-                    float mx0 = max3(s[0], s[1], s[2]), mx1 = max3(s[3], s[4], s[5]);
-#pragma unroll
-                    for (int j = 6; j < 62; j += 4) {
-                        mx0 = max3(mx0, s[j], s[j + 1]);
-                        mx1 = max3(mx1, s[j + 2], s[j + 3]);
-                    }
-                    const float m_cand = max3(mx0, mx1, fmaxf(s[62], s[63])) * sl2;
+                if (any_mine) {                         // the same for both column halves of a row group
+                    float* xp = &ctl->x_part[x_n & 1u][0][0];
+                    xp[chalf * 128 + row] = m_loc;
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&ctl->x_ready[quad]);
+                    ok = mbar_wait(&ctl->x_ready[quad], x_n & 1u, ctl, p.status, 36);
+                    if (!ok) break;
+                    ++x_n;
+                    const float m_cand = fmaxf(m_loc, xp[(chalf ^ 1) * 128 + row]) * sl2;
                     const bool need = m_cand > m_ref + kRescaleThreshold;        // true on the first step (m_ref = -inf)
-                    rescale = __any_sync(0xffffffffu, need);
+                    const bool rescale = __any_sync(0xffffffffu, need);
                     if (need) {
                         alpha = ex2(m_ref - m_cand);
                         m_ref = m_cand;
                     }
-                    float sum0 = 0.f, sum1 = 0.f;
-                    const float neg_m = -m_ref;
-#pragma unroll
-                    for (int j = 0; j < 64; j += 2) {
-                        float t0, t1;
-                        ffma2(t0, t1, s[j], s[j + 1], sl2, neg_m);
-                        const float p0 = ex2(t0), p1 = ex2(t1);
-                        fadd2(sum0, sum1, p0, p1);
-                        pk[j >> 1] = pack_bf16(p0, p1);
-                    }
-                    l_sum = l_sum * alpha + (sum0 + sum1);
-                }
-                // P of the previous step must have been consumed, and O must be at rest, before touching either
-                ok = mbar_wait(&ctl->pv_done, (grp_n & 1u) ^ 1u, ctl, p.status, 32);
-                if (!ok) break;
-                tc_fence_after();
-                if (rescale && o_dirty) {
-#pragma unroll
-                    for (int half = 0; half < 2; ++half) {
-                        float o[32];
-                        tmem_ld32(lane_addr + kColO + half * 32, o);
+                    if (rescale && o_dirty) {           // this thread's 32 of the 64 accumulator columns
+                        tmem_ld32(lane_addr + kColO + chalf * 32, s);
                         tmem_wait_ld();
 #pragma unroll
-                        for (int j = 0; j < 32; j += 2) fmul2(o[j], o[j + 1], alpha);
-                        tmem_st32(lane_addr + kColO + half * 32, reinterpret_cast<unsigned*>(o));
+                        for (int t = 0; t < 32; t += 2) fmul2(s[t], s[t + 1], alpha);
+                        tmem_st32(lane_addr + kColO + chalf * 32, reinterpret_cast<unsigned*>(s));
                     }
                 }
-                if (full) {
-                    if (my_c >= 0) tmem_st32(lane_addr + kColP, pk);
-                    else tmem_st32_zero(lane_addr + kColP);                      // tile without a lower query block
-                } else {
-                    // split step: my probabilities go to my half, zeros to the half of the other key block
-                    if (my_c >= 0) tmem_st32(lane_addr + kColP + my_half * 32, pk);
-                    const int other_c = lower ? c0 : c1;
-                    if (other_c >= 0) tmem_st32_zero(lane_addr + kColP + (lower ? 0 : 32));
+                // ---- pass 2: probabilities of my columns; zeros for key blocks my half does not attend
+                float sum0 = 0.f, sum1 = 0.f;
+                const float neg_m = -m_ref;
+#pragma unroll 1
+                for (int j = 0; j < cnt; ++j) {
+                    const int who = e[j].who;
+                    if (who != kBothHalves && who != my_who) {                              // warp-uniform
+                        tmem_st16_zero(lane_addr + my_col + 64 * j);
+                        continue;
+                    }
+                    tmem_ld32(lane_addr + my_col + 64 * j, s);
+                    tmem_wait_ld();
+                    const unsigned kbo = (unsigned)(e[j].kb >> (chalf * 32));
+                    if (kbo != ~0u) {
+#pragma unroll
+                        for (int t = 0; t < 32; ++t) s[t] = ((kbo >> t) & 1u) ? s[t] : -INFINITY;
+                    }
+                    unsigned pk[16];
+#pragma unroll
+                    for (int t = 0; t < 32; t += 2) {
+                        float t0, t1;
+                        ffma2(t0, t1, s[t], s[t + 1], sl2, neg_m);
+                        const float p0 = ex2(t0), p1 = ex2(t1);
+                        fadd2(sum0, sum1, p0, p1);
+                        pk[t >> 1] = pack_bf16(p0, p1);
+                    }
+                    tmem_st16(lane_addr + my_col + 64 * j, pk);
                 }
+                l_sum = l_sum * alpha + (sum0 + sum1);
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
@@ -610,39 +671,39 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             }
             if (!ok) break;
             if (flags & kSegLast) {
-                // -------------------------------------------------------- epilogue of the tile
-                const int bh = slot->bh;
+                // -------------------------------------------------------- end of the tile: row sums, lse, output pointer
+                const int my_q = lower ? slot->qb : slot->qa;
                 const unsigned long long qbits = lower ? slot->qbits_b : slot->qbits_a;
                 const bool have = live && o_dirty;
+                float l_row = 0.f;
                 if (have) {
-                    ok = mbar_wait(&ctl->pv_done, (grp_n & 1u) ^ 1u, ctl, p.status, 33);   // last P V of the tile
+                    // the two column halves of a row add their sums
+                    float* lp = &ctl->l_part[epi_n & 1u][0][0];
+                    lp[chalf * 128 + row] = l_sum;
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&ctl->l_ready[quad]);
+                    ok = mbar_wait(&ctl->l_ready[quad], epi_n & 1u, ctl, p.status, 34);
                     if (!ok) break;
-                    tc_fence_after();
+                    l_row = l_sum + lp[(chalf ^ 1) * 128 + row];
+                    ++epi_n;
                 }
-                if (my_q >= 0) {
+                if (my_q >= 0) {                        // warp-uniform
                     const int r64 = row & (kBlock - 1);
-                    const bool good = have && ((qbits >> r64) & 1ull) && l_sum > 0.f;
-                    const float inv = good ? 1.f / l_sum : 0.f;
-                    const size_t tok = ((size_t)bh * p.nb + my_q) * kBlock + r64;
-                    uint4* dst = reinterpret_cast<uint4*>(p.out + tok * kBlock);
+                    const bool good = have && ((qbits >> r64) & 1ull) && l_row > 0.f;
+                    const size_t tok = ((size_t)slot->bh * p.nb + my_q) * kBlock + r64;
+                    uint4* dst = reinterpret_cast<uint4*>(p.out + tok * kBlock + chalf * 32);
+                    if (p.lse && chalf == 0) p.lse[tok] = good ? (m_ref + log2f(l_row)) * 0.6931471805599453f : -INFINITY;
+                    if (have) {
+                        // the accumulator is read when the next scores (or the end of work) say it is complete
+                        pend_out = true;
+                        pend_good = good;
+                        pend_inv = good ? 1.f / l_row : 0.f;
+                        pend_dst = dst;
+                    } else {
+                        const uint4 z = make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-                    for (int half = 0; half < 2; ++half) {
-                        float o[32];
-                        if (have) {                     // warp-uniform
-                            tmem_ld32(lane_addr + kColO + half * 32, o);
-                            tmem_wait_ld();
-                        }
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            uint4 v4;
-                            v4.x = good ? pack_bf16(o[8 * j + 0] * inv, o[8 * j + 1] * inv) : 0u;
-                            v4.y = good ? pack_bf16(o[8 * j + 2] * inv, o[8 * j + 3] * inv) : 0u;
-                            v4.z = good ? pack_bf16(o[8 * j + 4] * inv, o[8 * j + 5] * inv) : 0u;
-                            v4.w = good ? pack_bf16(o[8 * j + 6] * inv, o[8 * j + 7] * inv) : 0u;
-                            dst[half * 4 + j] = v4;
-                        }
+                        for (int j = 0; j < 4; ++j) dst[j] = z;
                     }
-                    if (p.lse) p.lse[tok] = good ? (m_ref + log2f(l_sum)) * 0.6931471805599453f : -INFINITY;
                 }
             }
             tc_fence_before();
@@ -662,6 +723,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     }
     tc_fence_after();
     if (warp == 1) {
+        __syncwarp();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
     if (threadIdx.x == 0) {

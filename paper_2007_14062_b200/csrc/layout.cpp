@@ -88,8 +88,8 @@ int build_layout_host(bigbird_layout* L, int chunk_steps) {
 
     // ---- tile schedule ----------------------------------------------------------------------------
     // Query blocks are stacked two by two into 2b-row tiles: the global blocks among themselves (every key
-    // block is a full step), the others in ascending order.  For a sparse tile the key blocks listed by both
-    // halves become full steps; the rest are zipped into split steps.
+    // block is attended by both halves), the others in ascending order.  A step is one key block together
+    // with the halves of the tile that attend it.
     std::vector<int> gq, sq;
     for (int j = 0; j < nb; ++j) (is_global[j] ? gq : sq).push_back(j);
     const int n_gtiles = ((int)gq.size() + 1) / 2, n_stiles = ((int)sq.size() + 1) / 2;
@@ -107,14 +107,14 @@ int build_layout_host(bigbird_layout* L, int chunk_steps) {
         L->split_tile_q.push_back(gq[2 * t]);
         L->split_tile_q.push_back(2 * t + 1 < (int)gq.size() ? gq[2 * t + 1] : kNoBlock);
     }
-    std::vector<int32_t> la, lb, pa, pb;
+    std::vector<int32_t> la, lb, both, pa, pb;
     for (int h = 0; h < H; ++h) {
         const int32_t base = (int32_t)L->steps.size();
         L->step_base.push_back(base);
         auto rel = [&]() { return (int32_t)L->steps.size() - base; };
         for (int t = 0; t < n_gtiles; ++t) {
             const int32_t begin = rel();
-            for (int c = 0; c < nb; ++c) L->steps.push_back(Step{c, kStepFull});
+            for (int c = 0; c < nb; ++c) L->steps.push_back(Step{c, kBothHalves});
             for (int p = 0; p < parts; ++p) {
                 Item it{};
                 it.qa = gq[2 * t];
@@ -138,22 +138,28 @@ int build_layout_host(bigbird_layout* L, int chunk_steps) {
             const int na = L->row_ptr[(size_t)h * nb + it.qa + 1] - L->row_ptr[(size_t)h * nb + it.qa];
             la.assign(ra, ra + na);
             if (it.qb == kNoBlock) {
-                for (int32_t c : la) L->steps.push_back(Step{c, kStepFull});
+                for (int32_t c : la) L->steps.push_back(Step{c, kBothHalves});
             } else {
                 const int32_t* rb = &L->col_idx[L->row_ptr[(size_t)h * nb + it.qb]];
                 const int nbk = L->row_ptr[(size_t)h * nb + it.qb + 1] - L->row_ptr[(size_t)h * nb + it.qb];
                 lb.assign(rb, rb + nbk);
+                both.clear();
                 pa.clear();
                 pb.clear();
                 size_t ia = 0, ib = 0;
                 while (ia < la.size() || ib < lb.size()) {                   // merge of two ascending lists
                     if (ib == lb.size() || (ia < la.size() && la[ia] < lb[ib])) pa.push_back(la[ia++]);
                     else if (ia == la.size() || lb[ib] < la[ia]) pb.push_back(lb[ib++]);
-                    else { L->steps.push_back(Step{la[ia], kStepFull}); ++ia; ++ib; }
+                    else { both.push_back(la[ia]); ++ia; ++ib; }
                 }
-                const size_t ns = std::max(pa.size(), pb.size());
-                for (size_t s = 0; s < ns; ++s)
-                    L->steps.push_back(Step{s < pa.size() ? pa[s] : kNoBlock, s < pb.size() ? pb[s] : kNoBlock});
+                // shared, upper-only and lower-only key blocks take turns, so that any run of three
+                // consecutive steps gives both halves of the tile about the same amount of work
+                const size_t ns = std::max(both.size(), std::max(pa.size(), pb.size()));
+                for (size_t s = 0; s < ns; ++s) {
+                    if (s < both.size()) L->steps.push_back(Step{both[s], kBothHalves});
+                    if (s < pa.size()) L->steps.push_back(Step{pa[s], kUpperHalf});
+                    if (s < pb.size()) L->steps.push_back(Step{pb[s], kLowerHalf});
+                }
             }
             it.step_count = rel() - it.step_begin;
             L->items.push_back(it);

@@ -7,13 +7,14 @@
 namespace bigbird {
 
 // One step of a tile's key sweep.  A tile stacks two query blocks (upper half = rows 0..b-1, lower half =
-// rows b..2b-1).  c1 == kStepFull: key block c0 is attended by both halves.  Otherwise the step is split:
-// the upper half attends key block c0 and the lower half key block c1 (either may be kNoBlock).
+// rows b..2b-1).  A step names one key block and which halves of the tile attend it.
 struct Step {
-    int32_t c0;
-    int32_t c1;
+    int32_t c;      // key block
+    int32_t who;    // kBothHalves, kUpperHalf or kLowerHalf
 };
-constexpr int32_t kStepFull = -2;
+constexpr int32_t kBothHalves = 0;
+constexpr int32_t kUpperHalf = 1;
+constexpr int32_t kLowerHalf = 2;
 constexpr int32_t kNoBlock = -1;
 
 // One unit of work for a CTA: a tile of two query blocks and a contiguous range of steps.

@@ -77,13 +77,10 @@ def test_schedule_covers_every_listed_pair_exactly_once(cfg):
             qa, qb, sbeg, scnt, part, nparts, tile, _ = (int(x) for x in it)
             assert 0 <= qa < nb and (qb == -1 or 0 <= qb < nb) and qa != qb
             for s in steps[base[h] + sbeg: base[h] + sbeg + scnt]:
-                c0, c1 = int(s[0]), int(s[1])
-                if c1 == -2:
-                    pairs = [(qa, c0)] + ([(qb, c0)] if qb >= 0 else [])
-                else:
-                    assert c0 >= 0 or c1 >= 0
-                    pairs = ([(qa, c0)] if c0 >= 0 else []) + ([(qb, c1)] if c1 >= 0 else [])
-                    assert qb >= 0 or c1 < 0
+                c, who = int(s[0]), int(s[1])
+                assert 0 <= c < nb and who in (0, 1, 2)
+                assert qb >= 0 or who == 0
+                pairs = ([(qa, c)] if who in (0, 1) else []) + ([(qb, c)] if who in (0, 2) and qb >= 0 else [])
                 for pr in pairs:
                     assert pr not in seen
                     seen[pr] = 1
