@@ -8,16 +8,16 @@
 //     The MMAs always cover all 128 rows; rows that do not attend a key block get probability zero for it.
 //   * A producer thread fetches Q once per tile and the K and V blocks with TMA (128-byte swizzle) straight
 //     from the [B, H, N, D] tensors into a shared-memory ring: nothing is gathered or packed in HBM.
-//   * Key blocks are processed three at a time (one "step").  Their K tiles land in three adjacent ring slots, so
+//   * Key blocks are processed up to three at a time (one "step").  Their K tiles land in three adjacent ring slots, so
 //     that S = Q K^T of a step is one N = 192 tcgen05.mma per 16 head dimensions (an MMA instruction costs its
 //     issuing thread about the same time whatever its N, so wide MMAs are the cheap ones).  O += P V follows
 //     with P read from tensor memory, where the bf16 probabilities of a block overwrite its own scores.
-//   * Eight softmax warps: two threads share a row, each owning 32 of the 64 score columns of a key block.
-//     Pass 1 finds the row maximum (the two threads exchange theirs through shared memory), pass 2 re-reads
-//     the scores, applies the key-padding mask, exponentiates (base 2, fp32), sums, and writes the
-//     probabilities back.  The accumulator is rescaled only when the running maximum grows by more than 2^8.
-//     The two partial row sums meet at the end of the tile.  The output of a tile is written while the first
-//     step of the next tile is already in flight.
+//   * Four softmax warps, one thread per row of the tile.  A step is cut so that no row attends more than two
+//     of its key blocks: the thread pulls its (up to) 128 scores into registers with tcgen05.ld, applies the
+//     key-padding mask, takes the row maximum, exponentiates (base 2, fp32), sums, and writes bf16
+//     probabilities back with tcgen05.st (zeros for key blocks its half of the tile does not attend).  The
+//     accumulator is rescaled only when the running maximum grows by more than 2^8.  The output of a tile is
+//     written while the first step of the next tile is already in flight.
 //   * CTAs are persistent and draw work from a global counter: global-row tiles first, then the sparse tiles
 //     in (batch, head)-major order.  Two CTAs share an SM so that one's softmax overlaps the other's MMAs.
 //
@@ -40,8 +40,15 @@ constexpr int kTileBytes = kBlock * kBlock * 2;      // one 64x64 bf16 tile
 constexpr int kStepChunks = 3;             // key blocks per step
 constexpr int kRingGroups = 3;             // ring of groups of kStepChunks adjacent tiles (the K or the V blocks of one step)
 constexpr int kGroupBytes = kStepChunks * kTileBytes;
-constexpr int kThreads = 384;              // warp 0 TMA, warp 1 MMA issuer, warp 2 scheduler, warp 3 idle, warps 4..11 softmax
-constexpr int kSoftmaxWarps = 8;
+constexpr int kThreads = 256;              // warp 0 TMA, warp 1 MMA issuer, warp 2 scheduler, warp 3 idle, warps 4..7 softmax
+constexpr int kSoftmaxWarps = 4;
+#ifndef BB_REGS_LIGHT
+#define BB_REGS_LIGHT 72
+#define BB_REGS_SOFTMAX 184
+#endif
+constexpr int kRegsLight = BB_REGS_LIGHT;             // registers per thread of warps 0..3 after setmaxnreg
+constexpr int kRegsSoftmax = BB_REGS_SOFTMAX;          // registers per thread of warps 4..7 after setmaxnreg
+constexpr int kRowChunks = 2;              // key blocks one row may attend in a step (their scores live in registers)
 constexpr int kTmemCols = 256;
 constexpr int kColS = 0;                   // kStepChunks x 64 fp32 score columns; a block's probabilities reuse its columns
 constexpr int kColO = kStepChunks * 64;    // output accumulator: 64 fp32 columns
@@ -63,9 +70,10 @@ struct __align__(16) WorkSlot {
     int bh, batch, qa, qb;
     int n_chunks;
     int flags;
-    int pad_;
+    int n_steps;
     unsigned long long qbits_a, qbits_b;
     ChunkEntry chunks[kSegChunks];
+    unsigned char step_end[kSegChunks];    // step s covers chunks [step_end[s-1], step_end[s])
 };
 
 struct __align__(16) SmemCtl {
@@ -73,11 +81,7 @@ struct __align__(16) SmemCtl {
     unsigned long long empty[kRingGroups];
     unsigned long long q_full, q_empty;
     unsigned long long s_full, p_full;
-    unsigned long long x_ready[4];         // per 32-row group: both column halves have posted their row maxima
-    unsigned long long l_ready[4];         // per 32-row group: both column halves have posted their row sums
     unsigned long long sched_full[kSchedSlots], sched_empty[kSchedSlots];
-    float x_part[2][2][128];               // [step parity][column half][row]
-    float l_part[2][2][128];               // [tile parity][column half][row]
     unsigned tmem_base;
     int abort_flag;
     WorkSlot slot[kSchedSlots];
@@ -195,6 +199,16 @@ constexpr unsigned kIdescPV = kIdescQK64 | (1u << 16);
     F(o+24), F(o+25), F(o+26), F(o+27), F(o+28), F(o+29), F(o+30), F(o+31)
 #define BB_OUT(i) "=r"(u[i])
 #define BB_IN(i) "r"(u[i])
+__device__ __forceinline__ void tmem_ld64(unsigned taddr, float* r) {
+    unsigned* u = reinterpret_cast<unsigned*>(r);
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x64.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, "
+        "%32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, "
+        "%48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];"
+        : BB_REP32(BB_OUT, 0), BB_REP32(BB_OUT, 32) : "r"(taddr) : "memory");
+}
 __device__ __forceinline__ void tmem_ld32(unsigned taddr, float* r) {
     unsigned* u = reinterpret_cast<unsigned*>(r);
     asm volatile(
@@ -227,6 +241,14 @@ __device__ __forceinline__ void tmem_st16(unsigned taddr, const unsigned* u) {
 }
 #undef BB_OUT
 #undef BB_IN
+__device__ __forceinline__ void tmem_st32_zero(unsigned taddr) {
+    const unsigned z = 0;
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%1], "
+        "{%0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, "
+        "%0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0};"
+        ::"r"(z), "r"(taddr) : "memory");
+}
 __device__ __forceinline__ void tmem_st16_zero(unsigned taddr) {
     const unsigned z = 0;
     asm volatile(
@@ -272,14 +294,16 @@ __device__ __forceinline__ unsigned long long key_bits(const KernelParams& p, in
     if (c < 0) return 0ull;
     return p.kbits ? p.kbits[(size_t)batch * p.nb + c] : ~0ull;
 }
-__device__ __forceinline__ float row_max32(const float* s) {
-    float mx0 = max3(s[0], s[1], s[2]), mx1 = max3(s[3], s[4], s[5]);
+__device__ __forceinline__ float row_max64(const float* s) {
+    float mx0 = max3(s[0], s[1], s[2]), mx1 = max3(s[3], s[4], s[5]), mx2 = max3(s[6], s[7], s[8]), mx3 = max3(s[9], s[10], s[11]);
 #pragma unroll
-    for (int j = 6; j < 30; j += 4) {
+    for (int j = 12; j < 60; j += 8) {
         mx0 = max3(mx0, s[j], s[j + 1]);
         mx1 = max3(mx1, s[j + 2], s[j + 3]);
+        mx2 = max3(mx2, s[j + 4], s[j + 5]);
+        mx3 = max3(mx3, s[j + 6], s[j + 7]);
     }
-    return max3(mx0, mx1, fmaxf(s[30], s[31]));
+    return fmaxf(max3(mx0, mx1, fmaxf(s[60], s[61])), max3(mx2, mx3, fmaxf(s[62], s[63])));
 }
 
 // ------------------------------------------------------------------------------------------------ the kernel
@@ -297,7 +321,6 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         mbar_init(&ctl->q_empty, 1);
         mbar_init(&ctl->s_full, 1);
         mbar_init(&ctl->p_full, kSoftmaxWarps);
-        for (int i = 0; i < 4; ++i) { mbar_init(&ctl->x_ready[i], 2); mbar_init(&ctl->l_ready[i], 2); }
         for (int i = 0; i < kSchedSlots; ++i) { mbar_init(&ctl->sched_full[i], 1); mbar_init(&ctl->sched_empty[i], 2 + kSoftmaxWarps); }
         ctl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -313,6 +336,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     const unsigned tmem = *(volatile unsigned*)&ctl->tmem_base;
 
     if (warp < 4) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsLight));
         if (warp == 2) {
             // ================================================================= scheduler: fetch work, post live key blocks
             unsigned sched_n = 0;
@@ -371,7 +395,23 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                         count += __popc(bal);
                         i0 += 32;
                     }
+                    __syncwarp();
                     if (lane == 0) {
+                        // cut the live key blocks into steps: at most kStepChunks blocks, at most kRowChunks per half
+                        int ns = 0, cu = 0, cl = 0, cn = 0;
+                        for (int i = 0; i < count; ++i) {
+                            const int who = slot->chunks[i].who;
+                            const int au = who != kLowerHalf, al = who != kUpperHalf;
+                            if (cn == kStepChunks || cu + au > kRowChunks || cl + al > kRowChunks) {
+                                slot->step_end[ns++] = (unsigned char)i;
+                                cu = cl = cn = 0;
+                            }
+                            cu += au;
+                            cl += al;
+                            ++cn;
+                        }
+                        if (cn) slot->step_end[ns++] = (unsigned char)count;
+                        slot->n_steps = ns;
                         slot->w = w;
                         slot->bh = bh;
                         slot->batch = batch;
@@ -411,7 +451,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                 const unsigned ss = sched_n % kSchedSlots, sp = (sched_n / kSchedSlots) & 1u;
                 if (!mbar_wait(&ctl->sched_full[ss], sp, ctl, p.status, 13)) break;
                 const WorkSlot* slot = &ctl->slot[ss];
-                const int w = slot->w, flags = slot->flags, bh = slot->bh, n = slot->n_chunks;
+                const int w = slot->w, flags = slot->flags, bh = slot->bh, n = slot->n_steps;
                 if (w >= 0 && (flags & kSegLive)) {
                     if (flags & kSegFirst) {
                         const int qa = slot->qa, qb = slot->qb;
@@ -422,15 +462,17 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                         if (qb >= 0) tma_load_tile(smem + kSmemQ + kTileBytes, &tm_q, (bh * p.nb + qb) * kBlock, &ctl->q_full);
                         ++q_n;
                     }
-                    for (int i = 0; i < n && ok; i += kStepChunks) {
+                    for (int st = 0, i = 0; st < n && ok; ++st) {
                         if (pend_n > 0) ok = load_group(&tm_v, pend_bh, pend_c, pend_n);
                         if (!ok) break;
-                        pend_n = min(kStepChunks, n - i);
+                        const int end = slot->step_end[st];
+                        pend_n = end - i;
 #pragma unroll
                         for (int j = 0; j < kStepChunks; ++j)
                             if (j < pend_n) pend_c[j] = slot->chunks[i + j].c;
                         pend_bh = bh;
                         ok = load_group(&tm_k, bh, pend_c, pend_n);
+                        i = end;
                     }
                 }
                 mbar_arrive(&ctl->sched_empty[ss]);
@@ -473,9 +515,8 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                     if (j < pend_n) {
 #pragma unroll
                         for (int kk = 0; kk < 4; ++kk) {
-                            // 16 keys per MMA.  Keys 0..31 of a block sit in packed columns 0..15 of its score columns,
-                            // keys 32..63 in columns 32..47 (each softmax thread writes inside its own score columns).
-                            const unsigned a_col = kColS + 64 * j + (kk >> 1) * 32 + (kk & 1) * 8;
+                            // 16 keys per MMA: 8 packed columns of P_j, which sits in the first 32 score columns of block j
+                            const unsigned a_col = kColS + 64 * j + kk * 8;
                             mma_ts(tmem + kColO, tmem + a_col, v_desc + (unsigned long long)((j * kTileBytes + kk * 2048) >> 4), kIdescPV,
                                    (j > 0 || kk > 0 || !pend_fresh) ? 1u : 0u);
                         }
@@ -492,10 +533,10 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                 const unsigned ss = sched_n % kSchedSlots, sp = (sched_n / kSchedSlots) & 1u;
                 if (!mbar_wait(&ctl->sched_full[ss], sp, ctl, p.status, 23)) break;
                 const WorkSlot* slot = &ctl->slot[ss];
-                const int w = slot->w, flags = slot->flags, n = slot->n_chunks;
+                const int w = slot->w, flags = slot->flags, n = slot->n_steps;
                 if (w >= 0 && (flags & kSegLive)) {
                     bool first = flags & kSegFirst;
-                    for (int i = 0; i < n && ok; i += kStepChunks) {
+                    for (int st = 0, i = 0; st < n && ok; ++st) {
                         // P V of the previous step first: the scores of this step overwrite its probabilities,
                         // and MMAs execute in issue order
                         ok = pending_pv();
@@ -505,7 +546,9 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                             if (!ok) break;
                             tc_fence_after();
                         }
-                        const int cnt = min(kStepChunks, n - i);
+                        const int end = slot->step_end[st];
+                        const int cnt = end - i;
+                        i = end;
                         ok = qk(cnt);
                         if (!ok) break;
                         tc_commit(&ctl->s_full);        // also says: every earlier P V has completed
@@ -528,46 +571,61 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             }
         }
     } else {
-        // ===================================================================== softmax + epilogue (256 threads)
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
+        // ===================================================================== softmax + epilogue (128 threads, one per row)
         const int quad = warp & 3;                      // tensor-memory lanes this warp may touch: 32*quad .. +31
-        const int chalf = (warp - 4) >> 2;              // which 32 of a key block's 64 score columns this thread owns
         const int row = quad * 32 + lane;               // row of the 128-row tile
         const bool lower = row >= kBlock;
         const int my_who = lower ? kLowerHalf : kUpperHalf;
         const unsigned lane_addr = tmem + ((unsigned)(quad * 32) << 16);
-        const unsigned my_col = kColS + chalf * 32;     // first of my score columns in key block 0 of a step
         const float sl2 = p.scale_log2;
-        unsigned sched_n = 0, grp_n = 0, x_n = 0, epi_n = 0;
+        unsigned sched_n = 0, grp_n = 0;
         bool ok = true;
-        float m_ref = -INFINITY, l_sum = 0.f;           // l_sum: this thread's columns only
+        float m_ref = -INFINITY, l_sum = 0.f;
         bool o_dirty = false;                           // has any P V been issued for this tile yet
         // output of the previous tile, written once its last P V is known to be complete
         bool pend_out = false, pend_good = false;
         float pend_inv = 0.f;
         uint4* pend_dst = nullptr;
-        auto write_out = [&]() {                        // this thread's 32 accumulator columns of its row
+        auto write_out = [&]() {                        // the 64 accumulator columns of this thread's row
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
-                float o[16];
-                tmem_ld16(lane_addr + kColO + chalf * 32 + c * 16, o);
+                float o[32];
+                tmem_ld32(lane_addr + kColO + c * 32, o);
                 tmem_wait_ld();
 #pragma unroll
-                for (int j = 0; j < 2; ++j) {
+                for (int j = 0; j < 4; ++j) {
                     uint4 v4;
                     v4.x = pend_good ? pack_bf16(o[8 * j + 0] * pend_inv, o[8 * j + 1] * pend_inv) : 0u;
                     v4.y = pend_good ? pack_bf16(o[8 * j + 2] * pend_inv, o[8 * j + 3] * pend_inv) : 0u;
                     v4.z = pend_good ? pack_bf16(o[8 * j + 4] * pend_inv, o[8 * j + 5] * pend_inv) : 0u;
                     v4.w = pend_good ? pack_bf16(o[8 * j + 6] * pend_inv, o[8 * j + 7] * pend_inv) : 0u;
-                    pend_dst[2 * c + j] = v4;
+                    pend_dst[4 * c + j] = v4;
                 }
             }
             pend_out = false;
+        };
+        // exponentials of 64 scores of one key block -> packed bf16 probabilities in its first 32 columns
+        auto exp_store = [&](const float* s, unsigned col, float neg_m, float& sum0, float& sum1) {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                unsigned pk[16];
+#pragma unroll
+                for (int t = 0; t < 32; t += 2) {
+                    float t0, t1;
+                    ffma2(t0, t1, s[32 * h + t], s[32 * h + t + 1], sl2, neg_m);
+                    const float p0 = ex2(t0), p1 = ex2(t1);
+                    fadd2(sum0, sum1, p0, p1);
+                    pk[t >> 1] = pack_bf16(p0, p1);
+                }
+                tmem_st16(lane_addr + col + 16 * h, pk);
+            }
         };
         while (ok) {
             const unsigned ss = sched_n % kSchedSlots, sp = (sched_n / kSchedSlots) & 1u;
             if (!mbar_wait(&ctl->sched_full[ss], sp, ctl, p.status, 30)) break;
             const WorkSlot* slot = &ctl->slot[ss];
-            const int w = slot->w, flags = slot->flags, n = slot->n_chunks;
+            const int w = slot->w, flags = slot->flags, n = slot->n_steps;
             if (w < 0) {
                 if (pend_out) {                         // warp-uniform
                     ok = mbar_wait(&ctl->s_full, grp_n & 1u, ctl, p.status, 35);
@@ -583,85 +641,75 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                 l_sum = 0.f;
                 o_dirty = false;
             }
-            for (int i = 0; i < n && ok; i += kStepChunks) {
+            for (int st = 0, i = 0; st < n && ok; ++st) {
                 const ChunkEntry* e = &slot->chunks[i];
-                const int cnt = min(kStepChunks, n - i);
+                const int end = slot->step_end[st];
+                const int cnt = end - i;
+                i = end;
+                // the (at most two) key blocks of this step that my half of the tile attends: positions j0 < j1
+                int j0 = -1, j1 = -1;
+#pragma unroll
+                for (int j = 0; j < kStepChunks; ++j) {
+                    if (j < cnt) {
+                        const int who = e[j].who;
+                        if (who == kBothHalves || who == my_who) {                          // warp-uniform
+                            if (j0 < 0) j0 = j; else j1 = j;
+                        }
+                    }
+                }
                 ok = mbar_wait(&ctl->s_full, grp_n & 1u, ctl, p.status, 31);
                 if (!ok) break;
                 tc_fence_after();
                 // every P V issued before this step's scores has completed: the accumulator is at rest
                 if (pend_out) write_out();              // warp-uniform
-                // ---- pass 1: maximum of my columns over the key blocks my half of the tile attends
-                float s[32];
-                float m_loc = -INFINITY;
-                bool any_mine = false;
-#pragma unroll 1
-                for (int j = 0; j < cnt; ++j) {
-                    const int who = e[j].who;
-                    if (who != kBothHalves && who != my_who) continue;                      // warp-uniform
-                    any_mine = true;
-                    tmem_ld32(lane_addr + my_col + 64 * j, s);
-                    tmem_wait_ld();
-                    const unsigned kbo = (unsigned)(e[j].kb >> (chalf * 32));
-                    if (kbo != ~0u) {
-#pragma unroll
-                        for (int t = 0; t < 32; ++t) s[t] = ((kbo >> t) & 1u) ? s[t] : -INFINITY;
-                    }
-                    m_loc = fmaxf(m_loc, row_max32(s));
-                }
+                float s[128];
                 float alpha = 1.f;
-                if (any_mine) {                         // the same for both column halves of a row group
-                    float* xp = &ctl->x_part[x_n & 1u][0][0];
-                    xp[chalf * 128 + row] = m_loc;
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&ctl->x_ready[quad]);
-                    ok = mbar_wait(&ctl->x_ready[quad], x_n & 1u, ctl, p.status, 36);
-                    if (!ok) break;
-                    ++x_n;
-                    const float m_cand = fmaxf(m_loc, xp[(chalf ^ 1) * 128 + row]) * sl2;
+                if (j0 >= 0) {
+                    tmem_ld64(lane_addr + kColS + 64 * j0, s);
+                    if (j1 >= 0) tmem_ld64(lane_addr + kColS + 64 * j1, s + 64);
+                    tmem_wait_ld();
+                    const unsigned long long kb0 = e[j0].kb;
+                    if (kb0 != ~0ull) {
+#pragma unroll
+                        for (int t = 0; t < 64; ++t) s[t] = ((kb0 >> t) & 1ull) ? s[t] : -INFINITY;
+                    }
+                    float m_loc = row_max64(s);
+                    if (j1 >= 0) {
+                        const unsigned long long kb1 = e[j1].kb;
+                        if (kb1 != ~0ull) {
+#pragma unroll
+                            for (int t = 0; t < 64; ++t) s[64 + t] = ((kb1 >> t) & 1ull) ? s[64 + t] : -INFINITY;
+                        }
+                        m_loc = fmaxf(m_loc, row_max64(s + 64));
+                    }
+                    const float m_cand = m_loc * sl2;
                     const bool need = m_cand > m_ref + kRescaleThreshold;        // true on the first step (m_ref = -inf)
                     const bool rescale = __any_sync(0xffffffffu, need);
                     if (need) {
                         alpha = ex2(m_ref - m_cand);
                         m_ref = m_cand;
                     }
-                    if (rescale && o_dirty) {           // this thread's 32 of the 64 accumulator columns
-                        tmem_ld32(lane_addr + kColO + chalf * 32, s);
-                        tmem_wait_ld();
+                    if (rescale && o_dirty) {
 #pragma unroll
-                        for (int t = 0; t < 32; t += 2) fmul2(s[t], s[t + 1], alpha);
-                        tmem_st32(lane_addr + kColO + chalf * 32, reinterpret_cast<unsigned*>(s));
+                        for (int c = 0; c < 4; ++c) {
+                            float o[16];
+                            tmem_ld16(lane_addr + kColO + c * 16, o);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int t = 0; t < 16; t += 2) fmul2(o[t], o[t + 1], alpha);
+                            tmem_st16(lane_addr + kColO + c * 16, reinterpret_cast<unsigned*>(o));
+                        }
                     }
+                    float sum0 = 0.f, sum1 = 0.f;
+                    const float neg_m = -m_ref;
+                    exp_store(s, kColS + 64 * j0, neg_m, sum0, sum1);
+                    if (j1 >= 0) exp_store(s + 64, kColS + 64 * j1, neg_m, sum0, sum1);
+                    l_sum = l_sum * alpha + (sum0 + sum1);
                 }
-                // ---- pass 2: probabilities of my columns; zeros for key blocks my half does not attend
-                float sum0 = 0.f, sum1 = 0.f;
-                const float neg_m = -m_ref;
-#pragma unroll 1
-                for (int j = 0; j < cnt; ++j) {
-                    const int who = e[j].who;
-                    if (who != kBothHalves && who != my_who) {                              // warp-uniform
-                        tmem_st16_zero(lane_addr + my_col + 64 * j);
-                        continue;
-                    }
-                    tmem_ld32(lane_addr + my_col + 64 * j, s);
-                    tmem_wait_ld();
-                    const unsigned kbo = (unsigned)(e[j].kb >> (chalf * 32));
-                    if (kbo != ~0u) {
+                // zeros for the key blocks my half does not attend
 #pragma unroll
-                        for (int t = 0; t < 32; ++t) s[t] = ((kbo >> t) & 1u) ? s[t] : -INFINITY;
-                    }
-                    unsigned pk[16];
-#pragma unroll
-                    for (int t = 0; t < 32; t += 2) {
-                        float t0, t1;
-                        ffma2(t0, t1, s[t], s[t + 1], sl2, neg_m);
-                        const float p0 = ex2(t0), p1 = ex2(t1);
-                        fadd2(sum0, sum1, p0, p1);
-                        pk[t >> 1] = pack_bf16(p0, p1);
-                    }
-                    tmem_st16(lane_addr + my_col + 64 * j, pk);
-                }
-                l_sum = l_sum * alpha + (sum0 + sum1);
+                for (int j = 0; j < kStepChunks; ++j)
+                    if (j < cnt && j != j0 && j != j1) tmem_st32_zero(lane_addr + kColS + 64 * j);
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
@@ -671,38 +719,26 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             }
             if (!ok) break;
             if (flags & kSegLast) {
-                // -------------------------------------------------------- end of the tile: row sums, lse, output pointer
+                // -------------------------------------------------------- end of the tile: lse, output pointer
                 const int my_q = lower ? slot->qb : slot->qa;
                 const unsigned long long qbits = lower ? slot->qbits_b : slot->qbits_a;
                 const bool have = live && o_dirty;
-                float l_row = 0.f;
-                if (have) {
-                    // the two column halves of a row add their sums
-                    float* lp = &ctl->l_part[epi_n & 1u][0][0];
-                    lp[chalf * 128 + row] = l_sum;
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&ctl->l_ready[quad]);
-                    ok = mbar_wait(&ctl->l_ready[quad], epi_n & 1u, ctl, p.status, 34);
-                    if (!ok) break;
-                    l_row = l_sum + lp[(chalf ^ 1) * 128 + row];
-                    ++epi_n;
-                }
                 if (my_q >= 0) {                        // warp-uniform
                     const int r64 = row & (kBlock - 1);
-                    const bool good = have && ((qbits >> r64) & 1ull) && l_row > 0.f;
+                    const bool good = have && ((qbits >> r64) & 1ull) && l_sum > 0.f;
                     const size_t tok = ((size_t)slot->bh * p.nb + my_q) * kBlock + r64;
-                    uint4* dst = reinterpret_cast<uint4*>(p.out + tok * kBlock + chalf * 32);
-                    if (p.lse && chalf == 0) p.lse[tok] = good ? (m_ref + log2f(l_row)) * 0.6931471805599453f : -INFINITY;
+                    uint4* dst = reinterpret_cast<uint4*>(p.out + tok * kBlock);
+                    if (p.lse) p.lse[tok] = good ? (m_ref + log2f(l_sum)) * 0.6931471805599453f : -INFINITY;
                     if (have) {
                         // the accumulator is read when the next scores (or the end of work) say it is complete
                         pend_out = true;
                         pend_good = good;
-                        pend_inv = good ? 1.f / l_row : 0.f;
+                        pend_inv = good ? 1.f / l_sum : 0.f;
                         pend_dst = dst;
                     } else {
                         const uint4 z = make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) dst[j] = z;
+                        for (int j = 0; j < 8; ++j) dst[j] = z;
                     }
                 }
             }
