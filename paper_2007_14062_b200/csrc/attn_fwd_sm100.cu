@@ -8,16 +8,17 @@
 //     The MMAs always cover all 128 rows; rows that do not attend a key block get probability zero for it.
 //   * A producer thread fetches Q once per tile and the K and V blocks with TMA (128-byte swizzle) straight
 //     from the [B, H, N, D] tensors into a shared-memory ring: nothing is gathered or packed in HBM.
-//   * Key blocks are processed up to three at a time (one "step").  Their K tiles land in three adjacent ring slots, so
-//     that S = Q K^T of a step is one N = 192 tcgen05.mma per 16 head dimensions (an MMA instruction costs its
-//     issuing thread about the same time whatever its N, so wide MMAs are the cheap ones).  O += P V follows
-//     with P read from tensor memory, where the bf16 probabilities of a block overwrite its own scores.
-//   * Four softmax warps, one thread per row of the tile.  A step is cut so that no row attends more than two
-//     of its key blocks: the thread pulls its (up to) 128 scores into registers with tcgen05.ld, applies the
-//     key-padding mask, takes the row maximum, exponentiates (base 2, fp32), sums, and writes bf16
-//     probabilities back with tcgen05.st (zeros for key blocks its half of the tile does not attend).  The
-//     accumulator is rescaled only when the running maximum grows by more than 2^8.  The output of a tile is
-//     written while the first step of the next tile is already in flight.
+//   * Key blocks are processed two at a time (one "step").  Their K tiles land in adjacent ring slots, so that
+//     S = Q K^T of a step is one N = 128 tcgen05.mma per 16 head dimensions (an MMA instruction costs its issuing
+//     thread about the same time whatever its N, so wide MMAs are the cheap ones).  O += P V follows with P read
+//     from tensor memory.
+//   * Four softmax warps, one thread per row of the tile: the thread pulls its (up to) 128 scores into registers
+//     with tcgen05.ld and hands the score columns back at once, so that the next step's Q K^T runs under this
+//     step's exponentials; it applies the key-padding mask, takes the row maximum, exponentiates (base 2, fp32),
+//     sums, and writes bf16 probabilities with tcgen05.st (zeros for key blocks its half of the tile does not
+//     attend); the previous step's P V runs under the first half of that.  The accumulator is rescaled only
+//     when the running maximum grows by more than 2^8.  The output of a tile is written during the first step
+//     of the next tile.
 //   * CTAs are persistent and draw work from a global counter: global-row tiles first, then the sparse tiles
 //     in (batch, head)-major order.  Two CTAs share an SM so that one's softmax overlaps the other's MMAs.
 //
@@ -37,8 +38,8 @@ namespace {
 // ------------------------------------------------------------------------------------------------ constants
 constexpr int kBlock = 64;                 // tokens per block (b) and head dimension (D)
 constexpr int kTileBytes = kBlock * kBlock * 2;      // one 64x64 bf16 tile
-constexpr int kStepChunks = 3;             // key blocks per step
-constexpr int kRingGroups = 3;             // ring of groups of kStepChunks adjacent tiles (the K or the V blocks of one step)
+constexpr int kStepChunks = 2;             // key blocks per step
+constexpr int kRingGroups = 4;             // ring of groups of kStepChunks adjacent tiles (the K or the V blocks of one step)
 constexpr int kGroupBytes = kStepChunks * kTileBytes;
 constexpr int kThreads = 256;              // warp 0 TMA, warp 1 MMA issuer, warp 2 scheduler, warp 3 idle, warps 4..7 softmax
 constexpr int kSoftmaxWarps = 4;
@@ -48,10 +49,10 @@ constexpr int kSoftmaxWarps = 4;
 #endif
 constexpr int kRegsLight = BB_REGS_LIGHT;             // registers per thread of warps 0..3 after setmaxnreg
 constexpr int kRegsSoftmax = BB_REGS_SOFTMAX;          // registers per thread of warps 4..7 after setmaxnreg
-constexpr int kRowChunks = 2;              // key blocks one row may attend in a step (their scores live in registers)
 constexpr int kTmemCols = 256;
-constexpr int kColS = 0;                   // kStepChunks x 64 fp32 score columns; a block's probabilities reuse its columns
-constexpr int kColO = kStepChunks * 64;    // output accumulator: 64 fp32 columns
+constexpr int kColS = 0;                   // scores: kStepChunks x 64 fp32 columns
+constexpr int kColP = kStepChunks * 64;    // probabilities: kStepChunks x 32 columns of packed bf16 pairs
+constexpr int kColO = kColP + kStepChunks * 32;   // output accumulator: 64 fp32 columns
 constexpr float kRescaleThreshold = 8.0f;  // in log2 units
 constexpr long long kWaitLimitCycles = 4000000000ll;   // about two seconds
 constexpr int kSchedSlots = 3;
@@ -70,24 +71,23 @@ struct __align__(16) WorkSlot {
     int bh, batch, qa, qb;
     int n_chunks;
     int flags;
-    int n_steps;
+    int pad_;
     unsigned long long qbits_a, qbits_b;
-    ChunkEntry chunks[kSegChunks];
-    unsigned char step_end[kSegChunks];    // step s covers chunks [step_end[s-1], step_end[s])
+    ChunkEntry chunks[kSegChunks];         // step s of the segment covers chunks [kStepChunks s, kStepChunks (s + 1))
 };
 
 struct __align__(16) SmemCtl {
     unsigned long long full[kRingGroups];
     unsigned long long empty[kRingGroups];
-    unsigned long long q_full, q_empty;
-    unsigned long long s_full, p_full;
+    unsigned long long q_full[2], q_empty[2];
+    unsigned long long s_full, s_free, p_full, pv_done;
     unsigned long long sched_full[kSchedSlots], sched_empty[kSchedSlots];
     unsigned tmem_base;
     int abort_flag;
     WorkSlot slot[kSchedSlots];
 };
 constexpr int kSmemQ = 0;
-constexpr int kSmemRing = 2 * kTileBytes;
+constexpr int kSmemRing = 4 * kTileBytes;              // two Q buffers of two tiles each come first
 constexpr int kSmemCtl = kSmemRing + kRingGroups * kGroupBytes;
 constexpr int kSmemBytes = kSmemCtl + (int)sizeof(SmemCtl) + 1024;   // + slack for the 1024-byte alignment
 
@@ -317,10 +317,11 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < kRingGroups; ++i) { mbar_init(&ctl->full[i], 1); mbar_init(&ctl->empty[i], 1); }
-        mbar_init(&ctl->q_full, 1);
-        mbar_init(&ctl->q_empty, 1);
+        for (int i = 0; i < 2; ++i) { mbar_init(&ctl->q_full[i], 1); mbar_init(&ctl->q_empty[i], 1); }
         mbar_init(&ctl->s_full, 1);
+        mbar_init(&ctl->s_free, kSoftmaxWarps);
         mbar_init(&ctl->p_full, kSoftmaxWarps);
+        mbar_init(&ctl->pv_done, 1);
         for (int i = 0; i < kSchedSlots; ++i) { mbar_init(&ctl->sched_full[i], 1); mbar_init(&ctl->sched_empty[i], 2 + kSoftmaxWarps); }
         ctl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -395,23 +396,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                         count += __popc(bal);
                         i0 += 32;
                     }
-                    __syncwarp();
                     if (lane == 0) {
-                        // cut the live key blocks into steps: at most kStepChunks blocks, at most kRowChunks per half
-                        int ns = 0, cu = 0, cl = 0, cn = 0;
-                        for (int i = 0; i < count; ++i) {
-                            const int who = slot->chunks[i].who;
-                            const int au = who != kLowerHalf, al = who != kUpperHalf;
-                            if (cn == kStepChunks || cu + au > kRowChunks || cl + al > kRowChunks) {
-                                slot->step_end[ns++] = (unsigned char)i;
-                                cu = cl = cn = 0;
-                            }
-                            cu += au;
-                            cl += al;
-                            ++cn;
-                        }
-                        if (cn) slot->step_end[ns++] = (unsigned char)count;
-                        slot->n_steps = ns;
                         slot->w = w;
                         slot->bh = bh;
                         slot->batch = batch;
@@ -432,10 +417,10 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             }
         } else if (warp == 0 && lane == 0) {
             // ================================================================= TMA producer
-            // Ring order = the order in which the MMA thread consumes groups: V of step i-1, then K of step i.
+            // Ring order = the order in which the MMA thread consumes groups: K of step i, then V of step i-1.
             unsigned ring_n = 0, q_n = 0, sched_n = 0;
             bool ok = true;
-            // the (up to three) blocks c[0..cnt) of K or V into the next group of adjacent ring slots
+            // the (up to two) blocks c[0..cnt) of K or V into the next group of adjacent ring slots
             auto load_group = [&](const CUtensorMap* tm, int bh, const int* c, int cnt) -> bool {
                 const unsigned g = ring_n % kRingGroups, ph = (ring_n / kRingGroups) & 1u;
                 if (!mbar_wait(&ctl->empty[g], ph ^ 1u, ctl, p.status, 10)) return false;
@@ -446,33 +431,34 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                 ++ring_n;
                 return true;
             };
-            int pend_n = 0, pend_bh = 0, pend_c[kStepChunks] = {0, 0, 0};
+            int pend_n = 0, pend_bh = 0, pend_c[kStepChunks] = {0, 0};
             while (ok) {
                 const unsigned ss = sched_n % kSchedSlots, sp = (sched_n / kSchedSlots) & 1u;
                 if (!mbar_wait(&ctl->sched_full[ss], sp, ctl, p.status, 13)) break;
                 const WorkSlot* slot = &ctl->slot[ss];
-                const int w = slot->w, flags = slot->flags, bh = slot->bh, n = slot->n_steps;
+                const int w = slot->w, flags = slot->flags, bh = slot->bh, n = slot->n_chunks;
                 if (w >= 0 && (flags & kSegLive)) {
                     if (flags & kSegFirst) {
                         const int qa = slot->qa, qb = slot->qb;
-                        ok = mbar_wait(&ctl->q_empty, (q_n & 1u) ^ 1u, ctl, p.status, 12);
+                        const unsigned qs = q_n & 1u;
+                        ok = mbar_wait(&ctl->q_empty[qs], ((q_n >> 1) & 1u) ^ 1u, ctl, p.status, 12);
                         if (!ok) break;
-                        mbar_expect_tx(&ctl->q_full, qb >= 0 ? 2 * kTileBytes : kTileBytes);
-                        tma_load_tile(smem + kSmemQ, &tm_q, (bh * p.nb + qa) * kBlock, &ctl->q_full);
-                        if (qb >= 0) tma_load_tile(smem + kSmemQ + kTileBytes, &tm_q, (bh * p.nb + qb) * kBlock, &ctl->q_full);
+                        mbar_expect_tx(&ctl->q_full[qs], qb >= 0 ? 2 * kTileBytes : kTileBytes);
+                        tma_load_tile(smem + kSmemQ + qs * 2 * kTileBytes, &tm_q, (bh * p.nb + qa) * kBlock, &ctl->q_full[qs]);
+                        if (qb >= 0) tma_load_tile(smem + kSmemQ + qs * 2 * kTileBytes + kTileBytes, &tm_q, (bh * p.nb + qb) * kBlock, &ctl->q_full[qs]);
                         ++q_n;
                     }
-                    for (int st = 0, i = 0; st < n && ok; ++st) {
-                        if (pend_n > 0) ok = load_group(&tm_v, pend_bh, pend_c, pend_n);
-                        if (!ok) break;
-                        const int end = slot->step_end[st];
-                        pend_n = end - i;
+                    for (int i = 0; i < n && ok; i += kStepChunks) {
+                        int c[kStepChunks];
+                        const int cnt = min(kStepChunks, n - i);
 #pragma unroll
-                        for (int j = 0; j < kStepChunks; ++j)
-                            if (j < pend_n) pend_c[j] = slot->chunks[i + j].c;
+                        for (int j = 0; j < kStepChunks; ++j) c[j] = j < cnt ? slot->chunks[i + j].c : 0;
+                        ok = load_group(&tm_k, bh, c, cnt);
+                        if (ok && pend_n > 0) ok = load_group(&tm_v, pend_bh, pend_c, pend_n);
+#pragma unroll
+                        for (int j = 0; j < kStepChunks; ++j) pend_c[j] = c[j];
+                        pend_n = cnt;
                         pend_bh = bh;
-                        ok = load_group(&tm_k, bh, pend_c, pend_n);
-                        i = end;
                     }
                 }
                 mbar_arrive(&ctl->sched_empty[ss]);
@@ -484,14 +470,14 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             }
         } else if (warp == 1 && lane == 0) {
             // ================================================================= MMA issuer
-            unsigned ring_n = 0, q_n = 0, sched_n = 0, pv_n = 0;
+            unsigned ring_n = 0, q_n = 0, sched_n = 0, grp_n = 0, pv_n = 0;   // grp_n: steps whose Q K^T was issued
             bool ok = true;
-            const unsigned long long q_desc = smem_desc_sw128(smem_u32(smem + kSmemQ));
-            auto qk = [&](int cnt) -> bool {            // S[:, 0 .. 64 cnt) = Q K^T with the K blocks of the next ring group
+            auto qk = [&](int cnt, unsigned qs) -> bool {   // S[:, 0 .. 64 cnt) = Q K^T with the K blocks of the next ring group
                 const unsigned g = ring_n % kRingGroups, ph = (ring_n / kRingGroups) & 1u;
                 if (!mbar_wait(&ctl->full[g], ph, ctl, p.status, 20)) return false;
                 tc_fence_after();
                 // the blocks of a group are adjacent: their 64 cnt rows form one K-major operand
+                const unsigned long long q_desc = smem_desc_sw128(smem_u32(smem + kSmemQ + qs * 2 * kTileBytes));
                 const unsigned long long k_desc = smem_desc_sw128(smem_u32(smem + kSmemRing + g * kGroupBytes));
                 const unsigned idesc = kIdescQK64 + ((unsigned)(cnt - 1) << 20);           // N = 64 cnt
 #pragma unroll
@@ -502,6 +488,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                 return true;
             };
             bool pend_fresh = false;                    // the pending P V is the first of its tile: it overwrites O
+            bool tile_fresh = false, q_unseen = false;
             int pend_n = 0;
             auto pending_pv = [&]() -> bool {           // O (+)= sum_j P_j V_j with the V blocks of the next ring group
                 if (pend_n == 0) return true;
@@ -514,15 +501,13 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                 for (int j = 0; j < kStepChunks; ++j) {
                     if (j < pend_n) {
 #pragma unroll
-                        for (int kk = 0; kk < 4; ++kk) {
-                            // 16 keys per MMA: 8 packed columns of P_j, which sits in the first 32 score columns of block j
-                            const unsigned a_col = kColS + 64 * j + kk * 8;
-                            mma_ts(tmem + kColO, tmem + a_col, v_desc + (unsigned long long)((j * kTileBytes + kk * 2048) >> 4), kIdescPV,
+                        for (int kk = 0; kk < 4; ++kk)  // 16 keys per MMA: 8 packed columns of P_j, two 8-row groups of V_j
+                            mma_ts(tmem + kColO, tmem + kColP + 32 * j + kk * 8, v_desc + (unsigned long long)((j * kTileBytes + kk * 2048) >> 4), kIdescPV,
                                    (j > 0 || kk > 0 || !pend_fresh) ? 1u : 0u);
-                        }
                     }
                 }
                 tc_commit(&ctl->empty[g]);
+                tc_commit(&ctl->pv_done);
                 ++ring_n;
                 ++pv_n;
                 pend_n = 0;
@@ -533,39 +518,51 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                 const unsigned ss = sched_n % kSchedSlots, sp = (sched_n / kSchedSlots) & 1u;
                 if (!mbar_wait(&ctl->sched_full[ss], sp, ctl, p.status, 23)) break;
                 const WorkSlot* slot = &ctl->slot[ss];
-                const int w = slot->w, flags = slot->flags, n = slot->n_steps;
+                const int w = slot->w, flags = slot->flags, n = slot->n_chunks;
                 if (w >= 0 && (flags & kSegLive)) {
-                    bool first = flags & kSegFirst;
-                    for (int st = 0, i = 0; st < n && ok; ++st) {
-                        // P V of the previous step first: the scores of this step overwrite its probabilities,
-                        // and MMAs execute in issue order
-                        ok = pending_pv();
-                        if (!ok) break;
-                        if (first) {
-                            ok = mbar_wait(&ctl->q_full, q_n & 1u, ctl, p.status, 24);
+                    if (flags & kSegFirst) {
+                        ++q_n;                          // this tile's Q sits in buffer (q_n - 1) & 1
+                        q_unseen = true;
+                        tile_fresh = true;
+                    }
+                    const unsigned qs = (q_n - 1) & 1u, qph = ((q_n - 1) >> 1) & 1u;
+                    for (int i = 0; i < n && ok; i += kStepChunks) {
+                        // the softmax threads must have pulled the previous scores out of tensor memory
+                        if (grp_n > 0) {
+                            ok = mbar_wait(&ctl->s_free, (grp_n - 1) & 1u, ctl, p.status, 25);
                             if (!ok) break;
-                            tc_fence_after();
                         }
-                        const int end = slot->step_end[st];
-                        const int cnt = end - i;
-                        i = end;
-                        ok = qk(cnt);
+                        if (q_unseen) {
+                            ok = mbar_wait(&ctl->q_full[qs], qph, ctl, p.status, 24);
+                            if (!ok) break;
+                            q_unseen = false;
+                        }
+                        tc_fence_after();
+                        const int cnt = min(kStepChunks, n - i);
+                        ok = qk(cnt, qs);
                         if (!ok) break;
-                        tc_commit(&ctl->s_full);        // also says: every earlier P V has completed
+                        tc_commit(&ctl->s_full);
+                        ++grp_n;
+                        // the previous step's P V goes behind this step's Q K^T
+                        ok = pending_pv();
                         pend_n = cnt;
-                        pend_fresh = first;
-                        first = false;
+                        pend_fresh = tile_fresh;
+                        tile_fresh = false;
                     }
                     if (!ok) break;
                     if (flags & kSegLast) {
-                        tc_commit(&ctl->q_empty);       // every Q K^T of the tile has been issued
-                        ++q_n;
+                        if (q_unseen) {                 // a tile without a live key block: its Q still has to land
+                            ok = mbar_wait(&ctl->q_full[qs], qph, ctl, p.status, 26);
+                            if (!ok) break;
+                            q_unseen = false;
+                        }
+                        tc_commit(&ctl->q_empty[qs]);   // every Q K^T of the tile has been issued
                     }
                 }
                 mbar_arrive(&ctl->sched_empty[ss]);
                 ++sched_n;
                 if (w < 0) {
-                    if (pend_n > 0 && pending_pv()) tc_commit(&ctl->s_full);   // the last tile's accumulator is complete
+                    pending_pv();
                     break;
                 }
             }
@@ -589,23 +586,23 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         uint4* pend_dst = nullptr;
         auto write_out = [&]() {                        // the 64 accumulator columns of this thread's row
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                float o[32];
-                tmem_ld32(lane_addr + kColO + c * 32, o);
+            for (int c = 0; c < 4; ++c) {
+                float o[16];
+                tmem_ld16(lane_addr + kColO + c * 16, o);
                 tmem_wait_ld();
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
+                for (int j = 0; j < 2; ++j) {
                     uint4 v4;
                     v4.x = pend_good ? pack_bf16(o[8 * j + 0] * pend_inv, o[8 * j + 1] * pend_inv) : 0u;
                     v4.y = pend_good ? pack_bf16(o[8 * j + 2] * pend_inv, o[8 * j + 3] * pend_inv) : 0u;
                     v4.z = pend_good ? pack_bf16(o[8 * j + 4] * pend_inv, o[8 * j + 5] * pend_inv) : 0u;
                     v4.w = pend_good ? pack_bf16(o[8 * j + 6] * pend_inv, o[8 * j + 7] * pend_inv) : 0u;
-                    pend_dst[4 * c + j] = v4;
+                    pend_dst[2 * c + j] = v4;
                 }
             }
             pend_out = false;
         };
-        // exponentials of 64 scores of one key block -> packed bf16 probabilities in its first 32 columns
+        // exponentials of the 64 scores of one key block -> packed bf16 probabilities
         auto exp_store = [&](const float* s, unsigned col, float neg_m, float& sum0, float& sum1) {
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
@@ -625,10 +622,10 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             const unsigned ss = sched_n % kSchedSlots, sp = (sched_n / kSchedSlots) & 1u;
             if (!mbar_wait(&ctl->sched_full[ss], sp, ctl, p.status, 30)) break;
             const WorkSlot* slot = &ctl->slot[ss];
-            const int w = slot->w, flags = slot->flags, n = slot->n_steps;
+            const int w = slot->w, flags = slot->flags, n = slot->n_chunks;
             if (w < 0) {
-                if (pend_out) {                         // warp-uniform
-                    ok = mbar_wait(&ctl->s_full, grp_n & 1u, ctl, p.status, 35);
+                if (pend_out) {                         // warp-uniform; the last P V of all
+                    ok = mbar_wait(&ctl->pv_done, (grp_n - 1) & 1u, ctl, p.status, 35);
                     if (!ok) break;
                     tc_fence_after();
                     write_out();
@@ -641,75 +638,79 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                 l_sum = 0.f;
                 o_dirty = false;
             }
-            for (int st = 0, i = 0; st < n && ok; ++st) {
+            for (int i = 0; i < n && ok; i += kStepChunks) {
                 const ChunkEntry* e = &slot->chunks[i];
-                const int end = slot->step_end[st];
-                const int cnt = end - i;
-                i = end;
-                // the (at most two) key blocks of this step that my half of the tile attends: positions j0 < j1
-                int j0 = -1, j1 = -1;
-#pragma unroll
-                for (int j = 0; j < kStepChunks; ++j) {
-                    if (j < cnt) {
-                        const int who = e[j].who;
-                        if (who == kBothHalves || who == my_who) {                          // warp-uniform
-                            if (j0 < 0) j0 = j; else j1 = j;
-                        }
-                    }
-                }
+                const int cnt = min(kStepChunks, n - i);
+                // which of the step's key blocks my half of the tile attends (warp-uniform)
+                const int who0 = e[0].who, who1 = cnt > 1 ? e[1].who : -1;
+                const bool mine0 = who0 == kBothHalves || who0 == my_who;
+                const bool mine1 = who1 == kBothHalves || who1 == my_who;
                 ok = mbar_wait(&ctl->s_full, grp_n & 1u, ctl, p.status, 31);
                 if (!ok) break;
                 tc_fence_after();
-                // every P V issued before this step's scores has completed: the accumulator is at rest
-                if (pend_out) write_out();              // warp-uniform
                 float s[128];
+                if (mine0) tmem_ld64(lane_addr + kColS, s);
+                if (mine1) tmem_ld64(lane_addr + kColS + 64, s + 64);
+                tmem_wait_ld();
+                // the score columns are free again: the next step's Q K^T may overwrite them
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&ctl->s_free);
                 float alpha = 1.f;
-                if (j0 >= 0) {
-                    tmem_ld64(lane_addr + kColS + 64 * j0, s);
-                    if (j1 >= 0) tmem_ld64(lane_addr + kColS + 64 * j1, s + 64);
-                    tmem_wait_ld();
-                    const unsigned long long kb0 = e[j0].kb;
-                    if (kb0 != ~0ull) {
+                bool rescale = false;
+                if (mine0 || mine1) {
+                    float m_loc = -INFINITY;
+                    if (mine0) {
+                        const unsigned long long kb = e[0].kb;
+                        if (kb != ~0ull) {
 #pragma unroll
-                        for (int t = 0; t < 64; ++t) s[t] = ((kb0 >> t) & 1ull) ? s[t] : -INFINITY;
+                            for (int t = 0; t < 64; ++t) s[t] = ((kb >> t) & 1ull) ? s[t] : -INFINITY;
+                        }
+                        m_loc = row_max64(s);
                     }
-                    float m_loc = row_max64(s);
-                    if (j1 >= 0) {
-                        const unsigned long long kb1 = e[j1].kb;
-                        if (kb1 != ~0ull) {
+                    if (mine1) {
+                        const unsigned long long kb = e[1].kb;
+                        if (kb != ~0ull) {
 #pragma unroll
-                            for (int t = 0; t < 64; ++t) s[64 + t] = ((kb1 >> t) & 1ull) ? s[64 + t] : -INFINITY;
+                            for (int t = 0; t < 64; ++t) s[64 + t] = ((kb >> t) & 1ull) ? s[64 + t] : -INFINITY;
                         }
                         m_loc = fmaxf(m_loc, row_max64(s + 64));
                     }
                     const float m_cand = m_loc * sl2;
                     const bool need = m_cand > m_ref + kRescaleThreshold;        // true on the first step (m_ref = -inf)
-                    const bool rescale = __any_sync(0xffffffffu, need);
+                    rescale = __any_sync(0xffffffffu, need);
                     if (need) {
                         alpha = ex2(m_ref - m_cand);
                         m_ref = m_cand;
                     }
-                    if (rescale && o_dirty) {
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            float o[16];
-                            tmem_ld16(lane_addr + kColO + c * 16, o);
-                            tmem_wait_ld();
-#pragma unroll
-                            for (int t = 0; t < 16; t += 2) fmul2(o[t], o[t + 1], alpha);
-                            tmem_st16(lane_addr + kColO + c * 16, reinterpret_cast<unsigned*>(o));
-                        }
-                    }
-                    float sum0 = 0.f, sum1 = 0.f;
-                    const float neg_m = -m_ref;
-                    exp_store(s, kColS + 64 * j0, neg_m, sum0, sum1);
-                    if (j1 >= 0) exp_store(s + 64, kColS + 64 * j1, neg_m, sum0, sum1);
-                    l_sum = l_sum * alpha + (sum0 + sum1);
                 }
-                // zeros for the key blocks my half does not attend
+                // the previous step's P V must be complete before its probabilities are overwritten or O is touched
+                if (grp_n > 0) {
+                    ok = mbar_wait(&ctl->pv_done, (grp_n - 1) & 1u, ctl, p.status, 32);
+                    if (!ok) break;
+                    tc_fence_after();
+                }
+                if (pend_out) write_out();              // warp-uniform: the previous tile's accumulator is complete
+                if (rescale && o_dirty) {
 #pragma unroll
-                for (int j = 0; j < kStepChunks; ++j)
-                    if (j < cnt && j != j0 && j != j1) tmem_st32_zero(lane_addr + kColS + 64 * j);
+                    for (int c = 0; c < 4; ++c) {
+                        float o[16];
+                        tmem_ld16(lane_addr + kColO + c * 16, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int t = 0; t < 16; t += 2) fmul2(o[t], o[t + 1], alpha);
+                        tmem_st16(lane_addr + kColO + c * 16, reinterpret_cast<unsigned*>(o));
+                    }
+                }
+                float sum0 = 0.f, sum1 = 0.f;
+                const float neg_m = -m_ref;
+                if (mine0) exp_store(s, kColP, neg_m, sum0, sum1);
+                else tmem_st32_zero(lane_addr + kColP);
+                if (cnt > 1) {
+                    if (mine1) exp_store(s + 64, kColP + 32, neg_m, sum0, sum1);
+                    else tmem_st32_zero(lane_addr + kColP + 32);
+                }
+                l_sum = l_sum * alpha + (sum0 + sum1);
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
@@ -730,7 +731,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                     uint4* dst = reinterpret_cast<uint4*>(p.out + tok * kBlock);
                     if (p.lse) p.lse[tok] = good ? (m_ref + log2f(l_sum)) * 0.6931471805599453f : -INFINITY;
                     if (have) {
-                        // the accumulator is read when the next scores (or the end of work) say it is complete
+                        // the accumulator is read once the tile's last P V is known to be complete
                         pend_out = true;
                         pend_good = good;
                         pend_inv = good ? 1.f / l_sum : 0.f;
