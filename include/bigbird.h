@@ -39,7 +39,8 @@ enum {
     BIGBIRD_EUNSUPPORTED = -2,  /* shape or dtype outside what the kernels implement */
     BIGBIRD_ECUDA = -3,         /* a CUDA call failed; see bigbird_last_cuda_error() */
     BIGBIRD_ETIMEOUT = -4,      /* a bounded wait inside a kernel expired (reported by bigbird_last_status) */
-    BIGBIRD_ENOMEM = -5
+    BIGBIRD_ENOMEM = -5,
+    BIGBIRD_ELIMIT = -6         /* the problem exceeds the fixed scratch of bigbird_attn_fwd_static */
 };
 
 enum { BIGBIRD_ITC = 0, BIGBIRD_ETC = 1 };
@@ -129,6 +130,40 @@ BIGBIRD_API int bigbird_attn_fwd(const void* q, const void* k, const void* v, co
 BIGBIRD_API int bigbird_attn_fwd_simt(const void* q, const void* k, const void* v, const bigbird_layout* layout,
                           const uint8_t* key_padding_mask, void* out, float* lse,
                           int B, int H, int64_t N, int D, int b, float scale, int dtype, void* stream);
+
+/*
+ * bigbird_attn_fwd_static -- bigbird_attn_fwd for callers that must not allocate device memory.  (The paper has
+ * no counterpart: this is a property of the library, not of the method.)
+ *
+ * bigbird_attn_fwd keeps its scratch (status and work-counter words, the packed key-padding bits, the device
+ * copy of the layout's schedule) in memory it obtains with cudaMalloc on first use.  Some callers cannot have
+ * that: code that runs where device allocation is forbidden or would stall everyone else -- inside a region
+ * whose memory is owned by a pool the application sized up front, in a latency-critical serving loop where an
+ * implicit device synchronisation is unacceptable, or in a process that has handed all remaining GPU memory to
+ * another component.  This entry point calls no cudaMalloc, cudaFree or other allocating routine.  Its scratch
+ * is one fixed array of about 1.4 MB that is part of the library image: every GPU that loads the library
+ * holds it until the process exits.
+ *
+ * Arguments, layouts, results and asynchrony are those of bigbird_attn_fwd, with these differences:
+ *   - BIGBIRD_BF16 with D == 64 and b == 64 only (the tensor-core kernel); anything else is BIGBIRD_EUNSUPPORTED;
+ *   - limits set by the fixed array: B * N/b <= 16384, H * (tiles per head) <= 8192 and at most 131072 schedule
+ *     steps summed over heads (bigbird_layout_schedule reports both); beyond them the call does nothing and
+ *     returns BIGBIRD_ELIMIT;
+ *   - the schedule of `layout` is copied from host to device on every call (two cudaMemcpyAsync on `stream`),
+ *     so `layout` must not be destroyed while the call is being enqueued;
+ *   - the first call on a device looks up the array's device address and sets a kernel attribute; make that
+ *     first call outside any stream capture;
+ *   - all calls on a device share the array, which keeps the contents of the last call: the entry point
+ *     re-initialises what must start at zero, but two calls whose kernels overlap on the GPU (different
+ *     streams, or different threads) race on it and give undefined results.  Serialise them;
+ *   - a bounded wait that expires inside the kernel is not reported by bigbird_last_status (that function reads
+ *     the allocated scratch of bigbird_attn_fwd), and bigbird_last_launch_count / bigbird_last_cuda_error are
+ *     not updated.
+ * Errors: BIGBIRD_EINVAL, BIGBIRD_EUNSUPPORTED, BIGBIRD_ELIMIT, BIGBIRD_ECUDA.
+ */
+BIGBIRD_API int bigbird_attn_fwd_static(const void* q, const void* k, const void* v, const bigbird_layout* layout,
+                            const uint8_t* key_padding_mask, void* out, float* lse,
+                            int B, int H, int64_t N, int D, int b, float scale, int dtype, void* stream);
 
 /*
  * bigbird_last_status -- synchronises `stream` and reads the device status word of the current device:

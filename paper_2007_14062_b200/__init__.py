@@ -15,6 +15,7 @@ from .binding import (  # noqa: F401
     Layout,
     bigbird_attn_fwd,
     bigbird_attn_fwd_simt,
+    bigbird_attn_fwd_static,
     bigbird_build_layout,
     bigbird_last_launch_count,
     bigbird_last_status,

@@ -49,13 +49,14 @@ def lib() -> C.CDLL:
     fwd = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i64, i32, i32, f32, i32, vp]
     L.bigbird_attn_fwd.argtypes = fwd
     L.bigbird_attn_fwd_simt.argtypes = fwd
+    L.bigbird_attn_fwd_static.argtypes = fwd
     L.bigbird_last_status.argtypes = [vp, C.POINTER(i32), C.POINTER(i32)]
     L.bigbird_last_cuda_error.argtypes = []
     L.bigbird_last_launch_count.argtypes = []
     L.bigbird_strerror.argtypes = [i32]
     L.bigbird_strerror.restype = C.c_char_p
     for name in ("bigbird_build_layout", "bigbird_layout_nnz", "bigbird_layout_export", "bigbird_layout_schedule",
-                 "bigbird_layout_destroy", "bigbird_attn_fwd", "bigbird_attn_fwd_simt", "bigbird_last_status",
+                 "bigbird_layout_destroy", "bigbird_attn_fwd", "bigbird_attn_fwd_simt", "bigbird_attn_fwd_static", "bigbird_last_status",
                  "bigbird_last_cuda_error", "bigbird_last_launch_count"):
         getattr(L, name).restype = i32
     _lib = L
@@ -154,6 +155,13 @@ def bigbird_attn_fwd(q, k, v, layout: Layout, key_padding_mask, out, lse, scale:
 
 def bigbird_attn_fwd_simt(q, k, v, layout: Layout, key_padding_mask, out, lse, scale: float, stream: Optional[int] = None) -> None:
     _fwd("bigbird_attn_fwd_simt", q, k, v, layout, key_padding_mask, out, lse, scale, stream)
+
+
+def bigbird_attn_fwd_static(q, k, v, layout: Layout, key_padding_mask, out, lse, scale: float, stream: Optional[int] = None) -> None:
+    """bigbird_attn_fwd for callers that must not allocate device memory: the library's scratch is a fixed array
+    inside the loaded module.  bf16, D == 64, b == 64 only; BigBirdError(-6) if the problem exceeds the array.
+    Calls on one device must not overlap on the GPU; make the first call on a device outside stream capture."""
+    _fwd("bigbird_attn_fwd_static", q, k, v, layout, key_padding_mask, out, lse, scale, stream)
 
 
 def bigbird_last_status(stream: Optional[int] = None) -> Tuple[int, int]:

@@ -28,6 +28,7 @@
 #include <cuda_runtime.h>
 
 #include <mutex>
+#include <vector>
 
 #include "kernels.h"
 #include "../../include/bigbird.h"
@@ -889,3 +890,127 @@ int launch_attn_fwd_sm100(const FwdArgs& a, const bigbird_layout& L, const Devic
 }
 
 }  // namespace bigbird
+
+// ------------------------------------------------------------------------------------------------ no-allocation entry point
+// bigbird_attn_fwd_static: the tensor-core forward for callers that must not allocate device memory (see
+// include/bigbird.h).  Everything bigbird_attn_fwd keeps in cudaMalloc'ed library scratch lives here in one
+// fixed array that is part of the loaded module: status and work-counter words, the packed key-padding bits,
+// and the device copy of the layout's tile schedule, which is re-sent on every call.
+namespace bigbird {
+namespace {
+
+constexpr size_t kStaticMaskWords = 16384;      // B * N/b
+constexpr size_t kStaticItems = 8192;           // H * tiles per head
+constexpr size_t kStaticSteps = 131072;         // (key block, halves) entries summed over heads
+constexpr size_t kStaticOffMask = 256;          // bytes 0..15: status[2], counter[2]
+constexpr size_t kStaticOffItems = kStaticOffMask + kStaticMaskWords * sizeof(unsigned long long);
+constexpr size_t kStaticOffSteps = kStaticOffItems + kStaticItems * sizeof(Item);
+constexpr size_t kStaticBytes = kStaticOffSteps + kStaticSteps * sizeof(Step);      // about 1.4 MB per GPU
+
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
+
+struct StaticDevice {
+    unsigned char* base = nullptr;              // device address of g_static_scratch on this device
+    int sm_count = 0;
+};
+std::mutex g_static_mu;
+StaticDevice g_static_dev[64];
+
+// Once per device, with that device current: the device address of the array (its name is only a host-side
+// stand-in in host code) and the kernel's shared-memory attribute.
+cudaError_t static_setup(int device, StaticDevice* out) {
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    StaticDevice& d = g_static_dev[device];
+    if (!d.base) {
+        void* ptr = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(attn_fwd_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e != cudaSuccess) return e;
+        int sms = 0;
+        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+        if (e != cudaSuccess) return e;
+        d.sm_count = sms;
+        d.base = (unsigned char*)ptr;
+    }
+    *out = d;
+    return cudaSuccess;
+}
+
+}  // namespace
+}  // namespace bigbird
+
+extern "C" int bigbird_attn_fwd_static(const void* q, const void* k, const void* v, const bigbird_layout* L,
+                                       const uint8_t* key_padding_mask, void* out, float* lse, int B, int H, int64_t N,
+                                       int D, int b, float scale, int dtype, void* stream_) {
+    using namespace bigbird;
+    if (!q || !k || !v || !L || !out) return BIGBIRD_EINVAL;
+    if (B < 1 || H < 1 || N < 1 || D < 1 || b < 1) return BIGBIRD_EINVAL;
+    if (L->N != N || L->b != b || L->H != H) return BIGBIRD_EINVAL;
+    if (dtype != BIGBIRD_BF16 || D != 64 || b != 64) return BIGBIRD_EUNSUPPORTED;
+    if ((((uintptr_t)q) | ((uintptr_t)k) | ((uintptr_t)v) | ((uintptr_t)out)) & 15) return BIGBIRD_EINVAL;
+    if (!(scale > 0.f) || !(scale < INFINITY)) return BIGBIRD_EINVAL;
+    const int64_t rows = (int64_t)B * H * N;
+    if (rows >= (1ll << 31) || (int64_t)B * H * L->items_per_head >= (1ll << 31)) return BIGBIRD_EUNSUPPORTED;
+    // the fixed scratch bounds the problem
+    const size_t words = (size_t)B * L->nb, n_items = L->items.size(), n_steps = L->steps.size();
+    if (words > kStaticMaskWords || n_items > kStaticItems || n_steps > kStaticSteps) return BIGBIRD_ELIMIT;
+
+    int device = 0;
+    cudaError_t e = cudaGetDevice(&device);
+    if (e != cudaSuccess) return BIGBIRD_ECUDA;
+    if (device < 0 || device >= 64) return BIGBIRD_EUNSUPPORTED;
+    StaticDevice sd;
+    if (static_setup(device, &sd) != cudaSuccess) return BIGBIRD_ECUDA;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    int* words4 = reinterpret_cast<int*>(sd.base);
+    unsigned long long* kbits_dev = reinterpret_cast<unsigned long long*>(sd.base + kStaticOffMask);
+    Item* items_dev = reinterpret_cast<Item*>(sd.base + kStaticOffItems);
+    Step* steps_dev = reinterpret_cast<Step*>(sd.base + kStaticOffSteps);
+
+    CUtensorMap tm_q, tm_k, tm_v;
+    if (!make_map(&tm_q, q, (uint64_t)rows) || !make_map(&tm_k, k, (uint64_t)rows) || !make_map(&tm_v, v, (uint64_t)rows))
+        return BIGBIRD_ECUDA;
+
+    // The array keeps what the last call left: status and work counter must start at zero, and the schedule of
+    // this call's layout replaces the previous one (step offsets made absolute, as the kernel expects).
+    e = cudaMemsetAsync(words4, 0, 16, stream);
+    if (e != cudaSuccess) return BIGBIRD_ECUDA;
+    static thread_local std::vector<Item> items_abs;            // host memory only
+    items_abs = L->items;
+    for (int h = 0; h < L->H; ++h)
+        for (int i = 0; i < L->items_per_head; ++i) items_abs[(size_t)h * L->items_per_head + i].step_begin += L->step_base[h];
+    e = cudaMemcpyAsync(items_dev, items_abs.data(), n_items * sizeof(Item), cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess && n_steps) e = cudaMemcpyAsync(steps_dev, L->steps.data(), n_steps * sizeof(Step), cudaMemcpyHostToDevice, stream);
+    if (e != cudaSuccess) return BIGBIRD_ECUDA;
+
+    const unsigned long long* kbits = nullptr;
+    if (key_padding_mask) {
+        const int threads = 256, blocks = (int)((words * 32 + threads - 1) / threads);
+        pack_mask_kernel<<<blocks, threads, 0, stream>>>(key_padding_mask, kbits_dev, (int)words);
+        if (cudaGetLastError() != cudaSuccess) return BIGBIRD_ECUDA;
+        kbits = kbits_dev;
+    }
+
+    KernelParams p{};
+    p.out = (__nv_bfloat16*)out;
+    p.lse = lse;
+    p.kbits = kbits;
+    p.items = items_dev;
+    p.steps = steps_dev;
+    p.status = words4;
+    p.counter = words4 + 2;
+    p.items_per_head = L->items_per_head;
+    p.heavy_per_head = L->heavy_items_per_head;
+    p.BH = B * H;
+    p.H = H;
+    p.nb = L->nb;
+    p.total_work = p.BH * L->items_per_head;
+    p.scale_log2 = scale * 1.4426950408889634f;
+    int grid = 2 * sd.sm_count;
+    if (grid > p.total_work) grid = p.total_work;
+    if (grid < 1) grid = 1;
+    attn_fwd_sm100_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tm_q, tm_k, tm_v, p);
+    if (cudaGetLastError() != cudaSuccess) return BIGBIRD_ECUDA;
+    return BIGBIRD_OK;
+}

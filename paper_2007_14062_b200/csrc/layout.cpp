@@ -218,6 +218,7 @@ const char* bigbird_strerror(int code) {
         case BIGBIRD_ECUDA: return "CUDA call failed";
         case BIGBIRD_ETIMEOUT: return "bounded device wait expired";
         case BIGBIRD_ENOMEM: return "out of memory";
+        case BIGBIRD_ELIMIT: return "problem exceeds the fixed scratch of the no-allocation entry point";
         default: return "unknown error";
     }
 }
