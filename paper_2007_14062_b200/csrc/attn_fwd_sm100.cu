@@ -63,10 +63,12 @@ static_assert(kColO + 64 <= kTmemCols && kSegChunks % kStepChunks == 0, "tensor-
 // A key block of a tile after the key-padding mask has been applied.
 struct __align__(16) ChunkEntry {
     int c;                         // key block
-    int who;                       // kBothHalves, kUpperHalf or kLowerHalf: the halves of the tile that attend it
+    int who;                       // bits 0..1: kBothHalves, kUpperHalf or kLowerHalf (the halves of the tile that attend it);
+                                   // bit 2 (kHasPadding): some of its keys are padding
     unsigned long long kb;         // valid-key bits (never 0: blocks that are entirely padding are dropped)
 };
 enum { kSegFirst = 1, kSegLast = 2, kSegLive = 4 };
+enum { kWhoMask = 3, kHasPadding = 4, kNoChunk = 3 };
 struct __align__(16) WorkSlot {
     int w;                         // work index, -1 = no more work
     int bh, batch, qa, qb;
@@ -388,8 +390,8 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                             const bool ua = s.who != kLowerHalf && qbits_a != 0ull;
                             const bool ub = s.who != kUpperHalf && qbits_b != 0ull;
                             e.c = s.c;
-                            e.who = (ua && ub) ? kBothHalves : (ua ? kUpperHalf : kLowerHalf);
                             e.kb = key_bits(p, batch, s.c);
+                            e.who = ((ua && ub) ? kBothHalves : (ua ? kUpperHalf : kLowerHalf)) | (e.kb != ~0ull ? kHasPadding : 0);
                             alive = e.kb != 0ull && (ua || ub);
                         }
                         const unsigned bal = __ballot_sync(0xffffffffu, alive);
@@ -603,20 +605,26 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             }
             pend_out = false;
         };
-        // exponentials of the 64 scores of one key block -> packed bf16 probabilities
-        auto exp_store = [&](const float* s, unsigned col, float neg_m, float& sum0, float& sum1) {
+        // -inf over the scores of padded keys of one key block, in tensor memory (s: 64 scratch registers)
+        auto mask_scores = [&](float* s, unsigned taddr, unsigned long long kb) {
+            tmem_ld64(taddr, s);
+            tmem_wait_ld();
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                unsigned pk[16];
+            for (int t = 0; t < 64; ++t) s[t] = ((kb >> t) & 1ull) ? s[t] : -INFINITY;
+            tmem_st32(taddr, reinterpret_cast<unsigned*>(s));
+            tmem_st32(taddr + 32, reinterpret_cast<unsigned*>(s + 32));
+            tmem_wait_st();
+        };
+        // exponentials of the 64 scores of one key block, packed in place: afterwards s[0..31] hold the bit
+        // patterns of the 32 words of bf16 probability pairs
+        auto exp_pack = [&](float* s, float neg_m, float& sum0, float& sum1) {
 #pragma unroll
-                for (int t = 0; t < 32; t += 2) {
-                    float t0, t1;
-                    ffma2(t0, t1, s[32 * h + t], s[32 * h + t + 1], sl2, neg_m);
-                    const float p0 = ex2(t0), p1 = ex2(t1);
-                    fadd2(sum0, sum1, p0, p1);
-                    pk[t >> 1] = pack_bf16(p0, p1);
-                }
-                tmem_st16(lane_addr + col + 16 * h, pk);
+            for (int t = 0; t < 64; t += 2) {
+                float t0, t1;
+                ffma2(t0, t1, s[t], s[t + 1], sl2, neg_m);
+                const float p0 = ex2(t0), p1 = ex2(t1);
+                fadd2(sum0, sum1, p0, p1);
+                s[t >> 1] = __uint_as_float(pack_bf16(p0, p1));
             }
         };
         while (ok) {
@@ -643,13 +651,19 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                 const ChunkEntry* e = &slot->chunks[i];
                 const int cnt = min(kStepChunks, n - i);
                 // which of the step's key blocks my half of the tile attends (warp-uniform)
-                const int who0 = e[0].who, who1 = cnt > 1 ? e[1].who : -1;
-                const bool mine0 = who0 == kBothHalves || who0 == my_who;
-                const bool mine1 = who1 == kBothHalves || who1 == my_who;
+                const int who0 = e[0].who, who1 = cnt > 1 ? e[1].who : kNoChunk;
+                const bool mine0 = (who0 & kWhoMask) == kBothHalves || (who0 & kWhoMask) == my_who;
+                const bool mine1 = (who1 & kWhoMask) == kBothHalves || (who1 & kWhoMask) == my_who;
                 ok = mbar_wait(&ctl->s_full, grp_n & 1u, ctl, p.status, 31);
                 if (!ok) break;
                 tc_fence_after();
                 float s[128];
+                // A key block with padded keys (rare: the one holding a sequence's end) gets -inf written over their
+                // scores in tensor memory first, so that the common path below carries no masking code at all.
+                if (__builtin_expect(((who0 | who1) & kHasPadding) != 0, 0)) {
+                    if (mine0 && (who0 & kHasPadding)) mask_scores(s, lane_addr + kColS, e[0].kb);
+                    if (mine1 && (who1 & kHasPadding)) mask_scores(s, lane_addr + kColS + 64, e[1].kb);
+                }
                 if (mine0) tmem_ld64(lane_addr + kColS, s);
                 if (mine1) tmem_ld64(lane_addr + kColS + 64, s + 64);
                 tmem_wait_ld();
@@ -661,22 +675,8 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                 bool rescale = false;
                 if (mine0 || mine1) {
                     float m_loc = -INFINITY;
-                    if (mine0) {
-                        const unsigned long long kb = e[0].kb;
-                        if (kb != ~0ull) {
-#pragma unroll
-                            for (int t = 0; t < 64; ++t) s[t] = ((kb >> t) & 1ull) ? s[t] : -INFINITY;
-                        }
-                        m_loc = row_max64(s);
-                    }
-                    if (mine1) {
-                        const unsigned long long kb = e[1].kb;
-                        if (kb != ~0ull) {
-#pragma unroll
-                            for (int t = 0; t < 64; ++t) s[64 + t] = ((kb >> t) & 1ull) ? s[64 + t] : -INFINITY;
-                        }
-                        m_loc = fmaxf(m_loc, row_max64(s + 64));
-                    }
+                    if (mine0) m_loc = row_max64(s);
+                    if (mine1) m_loc = fmaxf(m_loc, row_max64(s + 64));
                     const float m_cand = m_loc * sl2;
                     const bool need = m_cand > m_ref + kRescaleThreshold;        // true on the first step (m_ref = -inf)
                     rescale = __any_sync(0xffffffffu, need);
@@ -685,14 +685,19 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                         m_ref = m_cand;
                     }
                 }
+                // probabilities into registers first: the previous step's P V has this long to finish
+                float sum0 = 0.f, sum1 = 0.f;
+                const float neg_m = -m_ref;
+                if (mine0) exp_pack(s, neg_m, sum0, sum1);
+                if (mine1) exp_pack(s + 64, neg_m, sum0, sum1);
                 // the previous step's P V must be complete before its probabilities are overwritten or O is touched
                 if (grp_n > 0) {
                     ok = mbar_wait(&ctl->pv_done, (grp_n - 1) & 1u, ctl, p.status, 32);
                     if (!ok) break;
                     tc_fence_after();
                 }
-                if (pend_out) write_out();              // warp-uniform: the previous tile's accumulator is complete
-                if (rescale && o_dirty) {
+                if (__builtin_expect(pend_out, 0)) write_out();      // warp-uniform: the previous tile's accumulator is complete
+                if (__builtin_expect(rescale && o_dirty, 0)) {
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
                         float o[16];
@@ -703,12 +708,10 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                         tmem_st16(lane_addr + kColO + c * 16, reinterpret_cast<unsigned*>(o));
                     }
                 }
-                float sum0 = 0.f, sum1 = 0.f;
-                const float neg_m = -m_ref;
-                if (mine0) exp_store(s, kColP, neg_m, sum0, sum1);
+                if (mine0) tmem_st32(lane_addr + kColP, reinterpret_cast<unsigned*>(s));
                 else tmem_st32_zero(lane_addr + kColP);
                 if (cnt > 1) {
-                    if (mine1) exp_store(s + 64, kColP + 32, neg_m, sum0, sum1);
+                    if (mine1) tmem_st32(lane_addr + kColP + 32, reinterpret_cast<unsigned*>(s + 64));
                     else tmem_st32_zero(lane_addr + kColP + 32);
                 }
                 l_sum = l_sum * alpha + (sum0 + sum1);
