@@ -155,7 +155,7 @@ __device__ __forceinline__ bool mbar_wait_slow(unsigned long long* bar, unsigned
     }
 }
 __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned parity, SmemCtl* ctl, int* status, int code) {
-    if (mbar_try(bar, parity)) return true;
+    if (__builtin_expect(mbar_try(bar, parity), 1)) return true;
     return mbar_wait_slow(bar, parity, ctl, status, code);
 }
 
