@@ -147,8 +147,9 @@ BIGBIRD_API int bigbird_attn_fwd_simt(const void* q, const void* k, const void* 
  * Arguments, layouts, results and asynchrony are those of bigbird_attn_fwd, with these differences:
  *   - BIGBIRD_BF16 with D == 64 and b == 64 only (the tensor-core kernel); anything else is BIGBIRD_EUNSUPPORTED;
  *   - limits set by the fixed array: B * N/b <= 16384, H * (tiles per head) <= 8192 and at most 131072 schedule
- *     steps summed over heads (bigbird_layout_schedule reports both); beyond them the call does nothing and
- *     returns BIGBIRD_ELIMIT;
+ *     steps summed over heads (bigbird_layout_schedule reports both), and N/b <= 96 (longer sequences have
+ *     their global tiles split into parts whose partial results need scratch that grows with B * H); beyond
+ *     them the call does nothing and returns BIGBIRD_ELIMIT;
  *   - the schedule of `layout` is copied from host to device on every call (two cudaMemcpyAsync on `stream`),
  *     so `layout` must not be destroyed while the call is being enqueued;
  *   - the first call on a device looks up the array's device address and sets a kernel attribute; make that

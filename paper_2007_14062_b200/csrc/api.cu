@@ -44,9 +44,8 @@ int get_scratch(int device, DeviceScratch** out) {
 template <typename T>
 cudaError_t upload(T** dst, const void* src, size_t count) {
     *dst = nullptr;
-    if (count == 0) count = 1;
-    cudaError_t e = cudaMalloc((void**)dst, count * sizeof(T));
-    if (e != cudaSuccess) return e;
+    cudaError_t e = cudaMalloc((void**)dst, (count ? count : 1) * sizeof(T));
+    if (e != cudaSuccess || count == 0) return e;
     return cudaMemcpy(*dst, src, count * sizeof(T), cudaMemcpyHostToDevice);
 }
 
@@ -55,6 +54,7 @@ void free_device_layout(DeviceLayout& d) {
     cudaFree(d.col_idx);
     cudaFree(d.items);
     cudaFree(d.steps);
+    cudaFree(d.split_tile_q);
     d = DeviceLayout{};
 }
 
@@ -77,6 +77,7 @@ int get_device_layout(const bigbird_layout* L, int device, DeviceLayout* out) {
         if (e == cudaSuccess) e = upload(&d.col_idx, L->col_idx.data(), L->col_idx.size());
         if (e == cudaSuccess) e = upload(&d.items, items.data(), items.size());
         if (e == cudaSuccess) e = upload(&d.steps, L->steps.data(), L->steps.size());
+        if (e == cudaSuccess) e = upload(&d.split_tile_q, L->split_tile_q.data(), L->split_tile_q.size());
         if (e != cudaSuccess) { free_device_layout(d); return cuda_fail(e); }
         d.device = device;
     }

@@ -19,6 +19,9 @@
 //     attend); the previous step's P V runs under the first half of that.  The accumulator is rescaled only
 //     when the running maximum grows by more than 2^8.  The output of a tile is written during the first step
 //     of the next tile.
+//   * A global-row tile of a long sequence is cut along the keys into parts that are separate work items; each
+//     writes its unnormalised accumulator and (max, sum) per row to scratch, and a small merge kernel combines
+//     the parts in a fixed order.
 //   * CTAs are persistent and draw work from a global counter: global-row tiles first, then the sparse tiles
 //     in (batch, head)-major order.  Two CTAs share an SM so that one's softmax overlaps the other's MMAs.
 //
@@ -57,6 +60,7 @@ constexpr int kColO = kColP + kStepChunks * 32;   // output accumulator: 64 fp32
 constexpr float kRescaleThreshold = 8.0f;  // in log2 units
 constexpr long long kWaitLimitCycles = 4000000000ll;   // about two seconds
 constexpr int kSchedSlots = 3;
+constexpr int kPartialFloats = 128 * 64 + 2 * 128;   // one part of a split tile: O[128][64], max[128], sum[128]
 constexpr int kSegChunks = 96;             // live key blocks per posted segment of a tile (a multiple of kStepChunks)
 static_assert(kColO + 64 <= kTmemCols && kSegChunks % kStepChunks == 0, "tensor-memory and segment layout");
 
@@ -74,7 +78,7 @@ struct __align__(16) WorkSlot {
     int bh, batch, qa, qb;
     int n_chunks;
     int flags;
-    int pad_;
+    int part_slot;                 // >= 0: the tile is one part of a split tile and writes partial results there
     unsigned long long qbits_a, qbits_b;
     ChunkEntry chunks[kSegChunks];         // step s of the segment covers chunks [kStepChunks s, kStepChunks (s + 1))
 };
@@ -106,6 +110,8 @@ struct KernelParams {
     int BH, H, nb;
     int total_work;
     float scale_log2;
+    float* partials;                   // [BH * split_tiles_per_head * max_parts][kPartialFloats] or nullptr
+    int split_tiles_per_head, max_parts;
 };
 
 // ------------------------------------------------------------------------------------------------ PTX wrappers
@@ -409,6 +415,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                         slot->flags = (first ? kSegFirst : 0) | (i0 >= n_raw ? kSegLast : 0) | (tile_live ? kSegLive : 0);
                         slot->qbits_a = qbits_a;
                         slot->qbits_b = qbits_b;
+                        slot->part_slot = (w >= 0 && item.nparts > 1) ? ((bh * p.split_tiles_per_head + item.tile) * p.max_parts + item.part) : -1;
                     }
                     __threadfence_block();
                     __syncwarp();
@@ -584,7 +591,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         float m_ref = -INFINITY, l_sum = 0.f;
         bool o_dirty = false;                           // has any P V been issued for this tile yet
         // output of the previous tile, written once its last P V is known to be complete
-        bool pend_out = false, pend_good = false;
+        bool pend_out = false, pend_good = false, pend_partial = false;
         float pend_inv = 0.f;
         uint4* pend_dst = nullptr;
         auto write_out = [&]() {                        // the 64 accumulator columns of this thread's row
@@ -593,6 +600,12 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                 float o[16];
                 tmem_ld16(lane_addr + kColO + c * 16, o);
                 tmem_wait_ld();
+                if (pend_partial) {                     // one part of a split tile: the raw fp32 accumulator
+                    float4* d4 = reinterpret_cast<float4*>(pend_dst) + 4 * c;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) d4[j] = make_float4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+                    continue;
+                }
 #pragma unroll
                 for (int j = 0; j < 2; ++j) {
                     uint4 v4;
@@ -728,7 +741,18 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                 const int my_q = lower ? slot->qb : slot->qa;
                 const unsigned long long qbits = lower ? slot->qbits_b : slot->qbits_a;
                 const bool have = live && o_dirty;
-                if (my_q >= 0) {                        // warp-uniform
+                const int part_slot = slot->part_slot;
+                if (part_slot >= 0) {
+                    // one part of a split tile: (max, sum) now, the accumulator once its last P V is complete
+                    float* part = p.partials + (size_t)part_slot * kPartialFloats;
+                    part[128 * 64 + row] = have ? m_ref : -INFINITY;
+                    part[128 * 64 + 128 + row] = have ? l_sum : 0.f;
+                    if (have) {
+                        pend_out = true;
+                        pend_partial = true;
+                        pend_dst = reinterpret_cast<uint4*>(part + row * 64);
+                    }
+                } else if (my_q >= 0) {                 // warp-uniform
                     const int r64 = row & (kBlock - 1);
                     const bool good = have && ((qbits >> r64) & 1ull) && l_sum > 0.f;
                     const size_t tok = ((size_t)slot->bh * p.nb + my_q) * kBlock + r64;
@@ -737,6 +761,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                     if (have) {
                         // the accumulator is read once the tile's last P V is known to be complete
                         pend_out = true;
+                        pend_partial = false;
                         pend_good = good;
                         pend_inv = good ? 1.f / l_sum : 0.f;
                         pend_dst = dst;
@@ -777,6 +802,53 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             __threadfence();
         }
     }
+}
+
+// Combines the parts of the split tiles: one CTA per (batch*head, split tile), one thread per row.
+__global__ void __launch_bounds__(128)
+merge_split_tiles_kernel(const float* __restrict__ partials, const int* __restrict__ tile_q, const unsigned long long* __restrict__ kbits,
+                         __nv_bfloat16* __restrict__ out, float* __restrict__ lse, int H, int nb, int tiles_per_head, int nparts) {
+    const int tile = blockIdx.x % tiles_per_head, bh = blockIdx.x / tiles_per_head;
+    const int row = threadIdx.x, r64 = row & (kBlock - 1);
+    const int q = tile_q[2 * tile + (row >> 6)];
+    if (q < 0) return;
+    const unsigned long long qb = kbits ? kbits[(size_t)(bh / H) * nb + q] : ~0ull;
+    const float* base = partials + (size_t)(bh * tiles_per_head + tile) * nparts * kPartialFloats;
+    float m = -INFINITY;
+    for (int pt = 0; pt < nparts; ++pt) m = fmaxf(m, base[(size_t)pt * kPartialFloats + 128 * 64 + row]);
+    float acc[64];
+#pragma unroll
+    for (int j = 0; j < 64; ++j) acc[j] = 0.f;
+    float l = 0.f;
+    if (m > -INFINITY) {
+        for (int pt = 0; pt < nparts; ++pt) {            // fixed order: results do not depend on scheduling
+            const float* part = base + (size_t)pt * kPartialFloats;
+            const float lp = part[128 * 64 + 128 + row];
+            if (!(lp > 0.f)) continue;
+            const float wgt = exp2f(part[128 * 64 + row] - m);
+            l += wgt * lp;
+            const float4* o4 = reinterpret_cast<const float4*>(part + row * 64);
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                const float4 v = o4[j];
+                acc[4 * j] += wgt * v.x; acc[4 * j + 1] += wgt * v.y; acc[4 * j + 2] += wgt * v.z; acc[4 * j + 3] += wgt * v.w;
+            }
+        }
+    }
+    const bool good = ((qb >> r64) & 1ull) && l > 0.f;
+    const float inv = good ? 1.f / l : 0.f;
+    const size_t tok = ((size_t)bh * nb + q) * kBlock + r64;
+    uint4* dst = reinterpret_cast<uint4*>(out + tok * kBlock);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        uint4 v4;
+        v4.x = pack_bf16(acc[8 * j + 0] * inv, acc[8 * j + 1] * inv);
+        v4.y = pack_bf16(acc[8 * j + 2] * inv, acc[8 * j + 3] * inv);
+        v4.z = pack_bf16(acc[8 * j + 4] * inv, acc[8 * j + 5] * inv);
+        v4.w = pack_bf16(acc[8 * j + 6] * inv, acc[8 * j + 7] * inv);
+        dst[j] = v4;
+    }
+    if (lse) lse[tok] = good ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
 }
 
 // One 64-bit word per (batch, key block): bit t = key_padding_mask[batch, block*64 + t] != 0.
@@ -866,10 +938,26 @@ int launch_attn_fwd_sm100(const FwdArgs& a, const bigbird_layout& L, const Devic
         kbits = sc.kbits;
     }
 
+    const bool split = L.split_tiles_per_head > 0 && L.max_parts > 1;
+    if (split) {
+        const size_t need = (size_t)a.B * a.H * L.split_tiles_per_head * L.max_parts * kPartialFloats;
+        if (need > sc.partials_cap) {                    // grows only when a larger problem shows up
+            cudaFree(sc.partials);
+            sc.partials = nullptr;
+            sc.partials_cap = 0;
+            cudaError_t e = cudaMalloc(&sc.partials, need * sizeof(float));
+            if (e != cudaSuccess) { *cuda_err = e; return BIGBIRD_ECUDA; }
+            sc.partials_cap = need;
+        }
+    }
+
     KernelParams p{};
     p.out = (__nv_bfloat16*)a.out;
     p.lse = a.lse;
     p.kbits = kbits;
+    p.partials = split ? sc.partials : nullptr;
+    p.split_tiles_per_head = L.split_tiles_per_head;
+    p.max_parts = L.max_parts;
     p.items = dl.items;
     p.steps = dl.steps;
     p.counter = sc.counters + 2 * (sc.next_slot++ % kCounterSlots);
@@ -889,6 +977,13 @@ int launch_attn_fwd_sm100(const FwdArgs& a, const bigbird_layout& L, const Devic
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { *cuda_err = e; return BIGBIRD_ECUDA; }
     ++*launches;
+    if (split) {
+        merge_split_tiles_kernel<<<p.BH * L.split_tiles_per_head, 128, 0, a.stream>>>(sc.partials, dl.split_tile_q, kbits, p.out, p.lse, a.H,
+                                                                                     a.nb, L.split_tiles_per_head, L.max_parts);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) { *cuda_err = e; return BIGBIRD_ECUDA; }
+        ++*launches;
+    }
     return BIGBIRD_OK;
 }
 
@@ -958,6 +1053,7 @@ extern "C" int bigbird_attn_fwd_static(const void* q, const void* k, const void*
     // the fixed scratch bounds the problem
     const size_t words = (size_t)B * L->nb, n_items = L->items.size(), n_steps = L->steps.size();
     if (words > kStaticMaskWords || n_items > kStaticItems || n_steps > kStaticSteps) return BIGBIRD_ELIMIT;
+    if (L->max_parts > 1) return BIGBIRD_ELIMIT;    // split global tiles need scratch for their partial results
 
     int device = 0;
     cudaError_t e = cudaGetDevice(&device);

@@ -93,7 +93,9 @@ int build_layout_host(bigbird_layout* L, int chunk_steps) {
     std::vector<int> gq, sq;
     for (int j = 0; j < nb; ++j) (is_global[j] ? gq : sq).push_back(j);
     const int n_gtiles = ((int)gq.size() + 1) / 2, n_stiles = ((int)sq.size() + 1) / 2;
-    if (chunk_steps <= 0) chunk_steps = nb;                                  // default: global tiles not split
+    // default: a global tile of a long sequence is cut into parts of 32 key blocks, about the work of a few
+    // sparse tiles, so that it does not outlast everything else; up to 96 blocks it stays whole
+    if (chunk_steps <= 0) chunk_steps = nb <= 96 ? nb : 32;
     const int parts = (nb + chunk_steps - 1) / chunk_steps;
     L->max_parts = parts;
     L->split_tiles_per_head = parts > 1 ? n_gtiles : 0;

@@ -35,6 +35,7 @@ struct DeviceLayout {
     int32_t* col_idx = nullptr;
     Item* items = nullptr;
     Step* steps = nullptr;
+    int32_t* split_tile_q = nullptr;   // [split_tiles_per_head * 2]
 };
 
 }  // namespace bigbird

@@ -85,6 +85,8 @@ SMALL = [
     _small("bf16", 1, 1, 4, g=4, r=0),                          # every block global
     _small("bf16", 1, 2, 6, g=0, r=1),                          # no global block
     _small("bf16", 1, 1, 1, g=1, r=0),                          # a single block
+    _small("bf16", 1, 2, 131, lengths="fixed:7000"),            # long sequence: the global tile is split along the keys
+    _small("bf16", 2, 1, 100, g=3, r=2),                        # split global tiles, an unpaired global block
     _small("fp32", 2, 2, 10, lengths="ragged:64:640"),
     _small("fp32", 1, 2, 7, mode=1, g=1, r=2),
 ]
