@@ -36,7 +36,7 @@ NOMINAL_BF16_TFLOPS = 2250.0
 FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "hbm_gbs": 6650.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one attn_fwd_sm100_kernel launch on this workload, from the
 # ncu capture summarised in profiles/ (None until a capture exists for the current kernel).
-NCU_DRAM_BYTES_PER_LAUNCH = {"c2_base_itc_bf16": 251.1e6}
+NCU_DRAM_BYTES_PER_LAUNCH = {"c2_base_itc_bf16": 257.1e6}
 
 
 def measured_peaks():
@@ -109,26 +109,36 @@ def oracle_slices(wl, q, k, v, kpm, slices):
     from oracle import bigbird_oracle as O
     gr = O.Graph(wl.N, wl.b, wl.w, wl.g, wl.r, wl.seed, wl.H, wl.mode)
     t0 = time.perf_counter()
-    O.attention(q, k, v, gr, kpm, wl.scale, slices=slices)
-    return time.perf_counter() - t0
+    res = O.attention(q, k, v, gr, kpm, wl.scale, slices=slices)
+    return time.perf_counter() - t0, res
 
 
-def cpu_baseline(wl, pairs_per_batch, budget_s=12.0):
-    """Times the oracle, as it stands, on a bounded sample of (batch, head) slices of the workload."""
+def cpu_baseline(wl, pairs_per_batch, gpu_out=None, gpu_lse=None, budget_s=12.0):
+    """Times the oracle, as it stands, on a bounded sample of (batch, head) slices of the workload, and compares
+    the library's output for those slices (batch element 0 of the first input set) with it."""
     q, k, v = synth.make_qkv(wl, batch_limit=1)
     qn, kn, vn = (t.float().numpy() for t in (q, k, v))
     kpm = synth.key_padding_mask(wl)
     kp = None if kpm is None else kpm.numpy()
     flops_per_slice = pairs_per_batch / wl.H * 4.0 * wl.b * wl.b * wl.D
-    t1 = oracle_slices(wl, qn, kn, vn, kp, [(0, 0)])
+    t1, _ = oracle_slices(wl, qn, kn, vn, kp, [(0, 0)])
     n = int(max(1, min(wl.H - 1, budget_s / max(t1, 1e-3))))
     slices = [(0, 1 + i) for i in range(n)] if wl.H > 1 else [(0, 0)]
-    t = oracle_slices(wl, qn, kn, vn, kp, slices)
+    t, res = oracle_slices(wl, qn, kn, vn, kp, slices)
     cores = len(os.sched_getaffinity(0))
-    return {"value": flops_per_slice * len(slices) / t / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"{len(slices)} of {wl.B * wl.H} (batch, head) slices at full N={wl.N}, fp64 masked dense attention; "
-                      f"{t / len(slices):.3f} s per slice",
-            "seconds_per_slice": t / len(slices)}
+    out = {"value": flops_per_slice * len(slices) / t / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
+           "sample": f"{len(slices)} of {wl.B * wl.H} (batch, head) slices at full N={wl.N}, fp64 masked dense attention; "
+                     f"{t / len(slices):.3f} s per slice",
+           "seconds_per_slice": t / len(slices)}
+    if gpu_out is not None:
+        valid = np.ones(wl.N, dtype=bool) if kp is None else kp[0] != 0
+        eo = el = 0.0
+        for (bi, h), (wo, wlse) in res.items():
+            eo = max(eo, float(np.abs(gpu_out[h][valid] - wo[valid]).max()))
+            el = max(el, float(np.abs(gpu_lse[h][valid] - wlse[valid]).max()))
+        out["max_abs_err_out_vs_oracle"] = eo
+        out["max_abs_err_lse_vs_oracle"] = el
+    return out
 
 
 def run_reference(args, wl):
@@ -147,7 +157,7 @@ def run_reference(args, wl):
         oracle_slices(wl, qn, kn, vn, kp, [(0, i % wl.H)])
     t = 0.0
     for i in range(args.steps):
-        t += oracle_slices(wl, qn, kn, vn, kp, [(0, i % wl.H)])
+        t += oracle_slices(wl, qn, kn, vn, kp, [(0, i % wl.H)])[0]
     value = flops_per_slice * args.steps / t / 1e12
     cores = len(os.sched_getaffinity(0))
     sample = f"each step = 1 of {wl.B * wl.H} (batch, head) slices at full N={wl.N} (fp64 masked dense attention on the host)"
@@ -165,7 +175,7 @@ def run_reference(args, wl):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=3000)
+    ap.add_argument("--steps", type=int, default=4000)
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2_base_itc_bf16", choices=synth.ORDER)
@@ -175,7 +185,7 @@ def main():
     wl = synth.WORKLOADS[args.workload]
 
     if args.impl == "reference":
-        if args.steps == 3000:
+        if args.steps == 4000:
             args.steps, args.warmup = 12, 3
         run_reference(args, wl)
         return
@@ -288,11 +298,11 @@ def main():
         per_gpu = tflops / world
         e2e_tflops = world * flops_per_step / (e2e_ms / args.e2e_steps * 1e-3) / 1e12
         traffic = NCU_DRAM_BYTES_PER_LAUNCH.get(wl.name)
-        min_bytes = wl.B * wl.H * wl.N * (4 * wl.D * 2 + 4)
+        min_bytes = wl.B * wl.H * wl.N * (4 * wl.D * (2 if wl.dtype == 'bf16' else 4) + 4)
         line = {
             "metric": METRIC, "value": tflops, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16", "data": "synthetic",
+            "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
             "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "N": wl.N, "D": wl.D, "block": wl.b, "window_blocks": wl.w,
                        "global_blocks": wl.g, "random_blocks": wl.r, "mode": "ETC" if wl.mode else "ITC",
                        "attended_block_pairs_per_step": wl.B * pairs, "counted_gflop_per_step": flops_per_step / 1e9,
@@ -307,14 +317,17 @@ def main():
             "clocks": sampler.summary(),
             "roofline": {"bound": "tensor", "achieved": per_gpu, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                          "frac": per_gpu / peaks["bf16_tflops"], "traffic": traffic,
-                         "peak_source": f"{peaks['source']} bf16 burst", "kernel": "attn_fwd_sm100_kernel",
+                         "peak_source": f"{peaks['source']} bf16 burst", "kernel": "attn_fwd_sm100_kernel" if wl.dtype == "bf16" else "attn_fwd_simt_kernel",
                          "kernel_us": 1e3 * ms_per_step, "algorithmic_flops_per_launch": flops_per_step,
                          "min_hbm_bytes_per_launch": min_bytes,
                          "achieved_hbm_gbs_on_min_bytes": min_bytes / (ms_per_step * 1e-3) / 1e9,
                          "frac_of_sustained_peak": per_gpu / peaks["bf16_tflops_sustained"] if peaks["bf16_tflops_sustained"] else None},
         }
         if world == 1 and not args.no_cpu_baseline:
-            line["cpu_baseline"] = cpu_baseline(wl, pairs)
+            # batch element 0 of the first input set holds the workload's own (unrolled) tensors
+            step(0)
+            torch.cuda.synchronize()
+            line["cpu_baseline"] = cpu_baseline(wl, pairs, sets[0][4][0].float().cpu().numpy(), sets[0][5][0].cpu().numpy())
         print(json.dumps(line))
     if dist is not None:
         dist.barrier()
