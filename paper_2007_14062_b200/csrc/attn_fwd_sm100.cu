@@ -591,29 +591,29 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         float m_ref = -INFINITY, l_sum = 0.f;
         bool o_dirty = false;                           // has any P V been issued for this tile yet
         // output of the previous tile, written once its last P V is known to be complete
-        bool pend_out = false, pend_good = false, pend_partial = false;
+        bool pend_out = false, pend_partial = false;
         float pend_inv = 0.f;
         uint4* pend_dst = nullptr;
         auto write_out = [&]() {                        // the 64 accumulator columns of this thread's row
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                float o[16];
-                tmem_ld16(lane_addr + kColO + c * 16, o);
+            for (int c = 0; c < 2; ++c) {
+                float o[32];
+                tmem_ld32(lane_addr + kColO + c * 32, o);
                 tmem_wait_ld();
                 if (pend_partial) {                     // one part of a split tile: the raw fp32 accumulator
-                    float4* d4 = reinterpret_cast<float4*>(pend_dst) + 4 * c;
+                    float4* d4 = reinterpret_cast<float4*>(pend_dst) + 8 * c;
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) d4[j] = make_float4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
-                    continue;
-                }
+                    for (int j = 0; j < 8; ++j) d4[j] = make_float4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+                } else {                                // pend_inv is 0 for rows that must come out as zeros
 #pragma unroll
-                for (int j = 0; j < 2; ++j) {
-                    uint4 v4;
-                    v4.x = pend_good ? pack_bf16(o[8 * j + 0] * pend_inv, o[8 * j + 1] * pend_inv) : 0u;
-                    v4.y = pend_good ? pack_bf16(o[8 * j + 2] * pend_inv, o[8 * j + 3] * pend_inv) : 0u;
-                    v4.z = pend_good ? pack_bf16(o[8 * j + 4] * pend_inv, o[8 * j + 5] * pend_inv) : 0u;
-                    v4.w = pend_good ? pack_bf16(o[8 * j + 6] * pend_inv, o[8 * j + 7] * pend_inv) : 0u;
-                    pend_dst[2 * c + j] = v4;
+                    for (int j = 0; j < 4; ++j) {
+                        uint4 v4;
+                        v4.x = pack_bf16(o[8 * j + 0] * pend_inv, o[8 * j + 1] * pend_inv);
+                        v4.y = pack_bf16(o[8 * j + 2] * pend_inv, o[8 * j + 3] * pend_inv);
+                        v4.z = pack_bf16(o[8 * j + 4] * pend_inv, o[8 * j + 5] * pend_inv);
+                        v4.w = pack_bf16(o[8 * j + 6] * pend_inv, o[8 * j + 7] * pend_inv);
+                        pend_dst[4 * c + j] = v4;
+                    }
                 }
             }
             pend_out = false;
@@ -762,7 +762,6 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                         // the accumulator is read once the tile's last P V is known to be complete
                         pend_out = true;
                         pend_partial = false;
-                        pend_good = good;
                         pend_inv = good ? 1.f / l_sum : 0.f;
                         pend_dst = dst;
                     } else {
