@@ -105,6 +105,21 @@ class ClockSampler:
                 "samples": len(self.samples)}
 
 
+def max_over_ranks(values, dist, device):
+    """Every rank's timings -> the slowest rank's (the job is as slow as its slowest replica).  `dist` is
+    torch.distributed or None for a single process."""
+    if dist is None:
+        return [float(v) for v in values]
+    t = torch.tensor(list(values), device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def whole_job_value(per_replica_units, world, slowest_ms):
+    """Aggregate throughput of `world` replicas that each process `per_replica_units` per step."""
+    return world * per_replica_units / (slowest_ms * 1e-3)
+
+
 def oracle_slices(wl, q, k, v, kpm, slices):
     from oracle import bigbird_oracle as O
     gr = O.Graph(wl.N, wl.b, wl.w, wl.g, wl.r, wl.seed, wl.H, wl.mode)
@@ -286,15 +301,12 @@ def main():
     h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv)) + (0 if hm is None else hm.numel())
     d2h = ho.numel() * ho.element_size() + hl.numel() * 4
 
-    if dist is not None:
-        t = torch.tensor([ms, e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, e2e_ms = float(t[0]), float(t[1])
+    ms, e2e_ms = max_over_ranks([ms, e2e_ms], dist, dev)
 
     if rank == 0:
         peaks = measured_peaks()
         ms_per_step = ms / args.steps
-        tflops = world * flops_per_step / (ms_per_step * 1e-3) / 1e12
+        tflops = whole_job_value(flops_per_step, world, ms_per_step) / 1e12
         per_gpu = tflops / world
         e2e_tflops = world * flops_per_step / (e2e_ms / args.e2e_steps * 1e-3) / 1e12
         traffic = NCU_DRAM_BYTES_PER_LAUNCH.get(wl.name)
