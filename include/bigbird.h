@@ -116,7 +116,9 @@ BIGBIRD_API int bigbird_layout_destroy(bigbird_layout* layout);
  *
  * Supported: D == 64 and b == 64 for BIGBIRD_BF16; D in {32, 64, 128} and any b for BIGBIRD_FP32.
  * The first call on a device (and the first call with a larger B, N or a new layout) allocates device
- * scratch owned by the library; later calls allocate nothing.
+ * scratch owned by the library; later calls allocate nothing.  That scratch (packed mask bits, partial results
+ * of split global tiles) is per device: calls that use a key-padding mask or a layout with N/b > 96 must not
+ * overlap on the GPU with other such calls (put them on one stream).
  * Errors: BIGBIRD_EINVAL, BIGBIRD_EUNSUPPORTED, BIGBIRD_ECUDA, BIGBIRD_ENOMEM.  There is no CPU path.
  */
 BIGBIRD_API int bigbird_attn_fwd(const void* q, const void* k, const void* v, const bigbird_layout* layout,
@@ -172,6 +174,14 @@ BIGBIRD_API int bigbird_attn_fwd_static(const void* q, const void* k, const void
  * its outputs are invalid).  *detail (may be NULL) receives a code naming the wait.  Clears the word.
  */
 BIGBIRD_API int bigbird_last_status(void* stream, int* status, int* detail);
+
+/*
+ * bigbird_selftest_wait_expiry -- failure-detection self-test.  Enqueues a one-thread kernel that waits, with the
+ * helper and the limit the attention kernel uses (about two seconds), on a barrier nothing ever signals.  The wait
+ * gives up, the kernel returns normally, and the next bigbird_last_status reports BIGBIRD_ETIMEOUT with detail 99;
+ * the context stays usable.  Nothing traps, faults or hangs.
+ */
+BIGBIRD_API int bigbird_selftest_wait_expiry(void* stream);
 
 /* The cudaError_t of the last failed CUDA call made by the library on this thread (0 if none). */
 BIGBIRD_API int bigbird_last_cuda_error(void);

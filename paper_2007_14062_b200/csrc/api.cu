@@ -180,6 +180,17 @@ int bigbird_last_status(void* stream, int* status, int* detail) {
     return BIGBIRD_OK;
 }
 
+int bigbird_selftest_wait_expiry(void* stream) {
+    int device = 0;
+    cudaError_t e = cudaGetDevice(&device);
+    if (e != cudaSuccess) return bigbird::cuda_fail(e);
+    bigbird::DeviceScratch* sc = nullptr;
+    int rc = bigbird::get_scratch(device, &sc);
+    if (rc != BIGBIRD_OK) return rc;
+    e = bigbird::launch_wait_expiry_selftest(*sc, (cudaStream_t)stream);
+    return e == cudaSuccess ? BIGBIRD_OK : bigbird::cuda_fail(e);
+}
+
 int bigbird_last_cuda_error(void) { return bigbird::t_last_cuda_error; }
 int bigbird_last_launch_count(void) { return bigbird::t_last_launches; }
 

@@ -850,6 +850,21 @@ merge_split_tiles_kernel(const float* __restrict__ partials, const int* __restri
     if (lse) lse[tok] = good ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
 }
 
+// Self-test of the bounded wait: one thread waits on an mbarrier that nothing ever arrives on, with the same
+// helper and the same limit as the attention kernel; the wait gives up, records BIGBIRD_ETIMEOUT and the kernel
+// returns normally.
+__global__ void wait_expiry_selftest_kernel(int* status) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    SmemCtl* ctl = reinterpret_cast<SmemCtl*>(smem + kSmemCtl);
+    if (threadIdx.x == 0) {
+        mbar_init(&ctl->s_full, 1);
+        ctl->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_wait(&ctl->s_full, 0u, ctl, status, 99);
+    }
+}
+
 // One 64-bit word per (batch, key block): bit t = key_padding_mask[batch, block*64 + t] != 0.
 __global__ void pack_mask_kernel(const uint8_t* __restrict__ kpm, unsigned long long* __restrict__ kbits, int n_words) {
     const int word = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -893,6 +908,13 @@ bool make_map(CUtensorMap* tm, const void* base, uint64_t rows) {
 }
 
 }  // namespace
+
+cudaError_t launch_wait_expiry_selftest(DeviceScratch& sc, cudaStream_t stream) {
+    cudaError_t e = cudaFuncSetAttribute(wait_expiry_selftest_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    wait_expiry_selftest_kernel<<<1, 32, kSmemBytes, stream>>>(sc.status);
+    return cudaGetLastError();
+}
 
 int launch_attn_fwd_sm100(const FwdArgs& a, const bigbird_layout& L, const DeviceLayout& dl, DeviceScratch& sc,
                           int* launches, cudaError_t* cuda_err) {

@@ -40,4 +40,7 @@ cudaError_t launch_attn_fwd_simt(const FwdArgs& a, const DeviceLayout& dl, int* 
 int launch_attn_fwd_sm100(const FwdArgs& a, const bigbird_layout& L, const DeviceLayout& dl, DeviceScratch& sc,
                           int* launches, cudaError_t* cuda_err);
 
+// One-thread kernel whose bounded wait is left to expire (about two seconds); sets the device status word.
+cudaError_t launch_wait_expiry_selftest(DeviceScratch& sc, cudaStream_t stream);
+
 }  // namespace bigbird

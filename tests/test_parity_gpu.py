@@ -146,6 +146,19 @@ def test_two_runs_are_bit_identical():
     assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
 
 
+def test_bounded_wait_expires_with_a_status_and_the_context_stays_usable():
+    """A wait that nothing will ever satisfy gives up after its limit: the kernel returns, the status word says
+    BIGBIRD_ETIMEOUT (-4) with the code of the wait, reading it clears it, and the next forward call is fine."""
+    assert bb.bigbird_last_status() == (0, 0)
+    bb.bigbird_selftest_wait_expiry()
+    assert bb.bigbird_last_status() == (-4, 99)
+    assert bb.bigbird_last_status() == (0, 0)
+    wl = _small("bf16", 1, 2, 8)
+    q, k, v = synth.make_qkv(wl)
+    out, lse = _run(wl, q, k, v, None)
+    _compare(wl, q, k, v, None, out, lse, slices=None)
+
+
 # ------------------------------------------------------------------------------------------------ full-size workloads
 def _sample_slices(wl, n, seed=0):
     rng = np.random.default_rng(seed)
