@@ -328,8 +328,8 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         for (int i = 0; i < kRingGroups; ++i) { mbar_init(&ctl->full[i], 1); mbar_init(&ctl->empty[i], 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(&ctl->q_full[i], 1); mbar_init(&ctl->q_empty[i], 1); }
         mbar_init(&ctl->s_full, 1);
-        mbar_init(&ctl->s_free, kSoftmaxWarps);
-        mbar_init(&ctl->p_full, kSoftmaxWarps);
+        mbar_init(&ctl->s_free, kSoftmaxWarps * 32);    // every softmax thread arrives itself: cheaper than
+        mbar_init(&ctl->p_full, kSoftmaxWarps * 32);    // converging the warp and electing a lane
         mbar_init(&ctl->pv_done, 1);
         for (int i = 0; i < kSchedSlots; ++i) { mbar_init(&ctl->sched_full[i], 1); mbar_init(&ctl->sched_empty[i], 2 + kSoftmaxWarps); }
         ctl->abort_flag = 0;
@@ -682,8 +682,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                 tmem_wait_ld();
                 // the score columns are free again: the next step's Q K^T may overwrite them
                 tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&ctl->s_free);
+                mbar_arrive(&ctl->s_free);
                 float alpha = 1.f;
                 bool rescale = false;
                 if (mine0 || mine1) {
@@ -730,8 +729,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                 l_sum = l_sum * alpha + (sum0 + sum1);
                 tmem_wait_st();
                 tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&ctl->p_full);
+                mbar_arrive(&ctl->p_full);
                 ++grp_n;
                 o_dirty = true;
             }
