@@ -161,9 +161,10 @@ def run_reference(args, wl):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    import paper_2007_14062_b200 as bb
-    L = bb.bigbird_build_layout(wl.N, wl.b, wl.w, wl.g, wl.r, wl.seed, wl.H, wl.mode)
-    flops_per_slice = counted_pairs(L, wl) / wl.H * 4.0 * wl.b * wl.b * wl.D
+    from oracle import bigbird_oracle as O
+    # attended block pairs counted from the oracle's own mask: nothing of the CUDA library is on this arm
+    row_ptr, _ = O.layout_from_mask(O.Graph(wl.N, wl.b, wl.w, wl.g, wl.r, wl.seed, wl.H, wl.mode))
+    flops_per_slice = int(row_ptr[-1]) / wl.H * 4.0 * wl.b * wl.b * wl.D
     q, k, v = synth.make_qkv(wl, batch_limit=1)
     qn, kn, vn = (t.float().numpy() for t in (q, k, v))
     kpm = synth.key_padding_mask(wl)
