@@ -801,21 +801,20 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     }
 }
 
-// Combines the parts of the split tiles: one CTA per (batch*head, split tile), one thread per row.
-__global__ void __launch_bounds__(128)
+// Combines the parts of the split tiles: one CTA per (batch*head, split tile, group of 16 rows); 16 threads share
+// a row, each owning 4 of its 64 output columns.
+__global__ void __launch_bounds__(256)
 merge_split_tiles_kernel(const float* __restrict__ partials, const int* __restrict__ tile_q, const unsigned long long* __restrict__ kbits,
                          __nv_bfloat16* __restrict__ out, float* __restrict__ lse, int H, int nb, int tiles_per_head, int nparts) {
-    const int tile = blockIdx.x % tiles_per_head, bh = blockIdx.x / tiles_per_head;
-    const int row = threadIdx.x, r64 = row & (kBlock - 1);
+    const int rgrp = blockIdx.x & 7, tile = (blockIdx.x >> 3) % tiles_per_head, bh = (blockIdx.x >> 3) / tiles_per_head;
+    const int row = rgrp * 16 + (threadIdx.x >> 4), c4 = threadIdx.x & 15, r64 = row & (kBlock - 1);
     const int q = tile_q[2 * tile + (row >> 6)];
     if (q < 0) return;
     const unsigned long long qb = kbits ? kbits[(size_t)(bh / H) * nb + q] : ~0ull;
     const float* base = partials + (size_t)(bh * tiles_per_head + tile) * nparts * kPartialFloats;
     float m = -INFINITY;
     for (int pt = 0; pt < nparts; ++pt) m = fmaxf(m, base[(size_t)pt * kPartialFloats + 128 * 64 + row]);
-    float acc[64];
-#pragma unroll
-    for (int j = 0; j < 64; ++j) acc[j] = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float l = 0.f;
     if (m > -INFINITY) {
         for (int pt = 0; pt < nparts; ++pt) {            // fixed order: results do not depend on scheduling
@@ -824,28 +823,18 @@ merge_split_tiles_kernel(const float* __restrict__ partials, const int* __restri
             if (!(lp > 0.f)) continue;
             const float wgt = exp2f(part[128 * 64 + row] - m);
             l += wgt * lp;
-            const float4* o4 = reinterpret_cast<const float4*>(part + row * 64);
-#pragma unroll
-            for (int j = 0; j < 16; ++j) {
-                const float4 v = o4[j];
-                acc[4 * j] += wgt * v.x; acc[4 * j + 1] += wgt * v.y; acc[4 * j + 2] += wgt * v.z; acc[4 * j + 3] += wgt * v.w;
-            }
+            const float4 v = reinterpret_cast<const float4*>(part + row * 64)[c4];
+            acc.x += wgt * v.x; acc.y += wgt * v.y; acc.z += wgt * v.z; acc.w += wgt * v.w;
         }
     }
     const bool good = ((qb >> r64) & 1ull) && l > 0.f;
     const float inv = good ? 1.f / l : 0.f;
     const size_t tok = ((size_t)bh * nb + q) * kBlock + r64;
-    uint4* dst = reinterpret_cast<uint4*>(out + tok * kBlock);
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        uint4 v4;
-        v4.x = pack_bf16(acc[8 * j + 0] * inv, acc[8 * j + 1] * inv);
-        v4.y = pack_bf16(acc[8 * j + 2] * inv, acc[8 * j + 3] * inv);
-        v4.z = pack_bf16(acc[8 * j + 4] * inv, acc[8 * j + 5] * inv);
-        v4.w = pack_bf16(acc[8 * j + 6] * inv, acc[8 * j + 7] * inv);
-        dst[j] = v4;
-    }
-    if (lse) lse[tok] = good ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
+    uint2 v2;
+    v2.x = pack_bf16(acc.x * inv, acc.y * inv);
+    v2.y = pack_bf16(acc.z * inv, acc.w * inv);
+    reinterpret_cast<uint2*>(out + tok * kBlock)[c4] = v2;
+    if (lse && c4 == 0) lse[tok] = good ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
 }
 
 // Self-test of the bounded wait: one thread waits on an mbarrier that nothing ever arrives on, with the same
@@ -997,7 +986,7 @@ int launch_attn_fwd_sm100(const FwdArgs& a, const bigbird_layout& L, const Devic
     if (e != cudaSuccess) { *cuda_err = e; return BIGBIRD_ECUDA; }
     ++*launches;
     if (split) {
-        merge_split_tiles_kernel<<<p.BH * L.split_tiles_per_head, 128, 0, a.stream>>>(sc.partials, dl.split_tile_q, kbits, p.out, p.lse, a.H,
+        merge_split_tiles_kernel<<<p.BH * L.split_tiles_per_head * 8, 256, 0, a.stream>>>(sc.partials, dl.split_tile_q, kbits, p.out, p.lse, a.H,
                                                                                      a.nb, L.split_tiles_per_head, L.max_parts);
         e = cudaGetLastError();
         if (e != cudaSuccess) { *cuda_err = e; return BIGBIRD_ECUDA; }
