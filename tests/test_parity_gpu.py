@@ -174,6 +174,27 @@ def test_c2_base_itc_bf16_full_size():
     _compare(wl, q, k, v, None, out, lse, slices=_sample_slices(wl, 6) + [(0, 0), (wl.B - 1, wl.H - 1)])
 
 
+def test_c2_full_size_closed_forms():
+    """Properties that hold at any size, on the full BigBird-base workload: V == 1 gives out == 1 everywhere;
+    Q == 0 gives lse = ln(64 * attended key blocks) per row, and the block counts are those of the layout."""
+    wl = synth.WORKLOADS["c2_base_itc_bf16"]
+    q, k, v = synth.make_qkv(wl)
+    out, _ = _run(wl, q, k, torch.ones_like(v), None)
+    assert np.abs(out - 1).max() <= 2 ** -8
+    out, lse = _run(wl, torch.zeros_like(q), k, v, None)
+    L = bb.bigbird_build_layout(wl.N, wl.b, wl.w, wl.g, wl.r, wl.seed, wl.H, wl.mode)
+    rp, _ = L.export()
+    blocks = np.diff(rp).reshape(wl.H, wl.nb)                      # attended key blocks per (head, query block)
+    want = np.log(64.0 * np.repeat(blocks, 64, axis=1))            # [H, N]
+    assert np.abs(lse - want[None]).max() < 1e-4
+    L.close()
+    # a key block permuted inside itself, jointly in K and V, changes nothing
+    perm = torch.arange(wl.N).reshape(wl.nb, 64)[:, torch.randperm(64, generator=torch.Generator().manual_seed(0))].reshape(-1)
+    a, la = _run(wl, q, k, v, None)
+    b2, lb = _run(wl, q, k[:, :, perm], v[:, :, perm], None)
+    assert np.abs(a - b2).max() <= 2e-2 and np.abs(la - lb).max() <= 1e-4
+
+
 def test_c3_etc_bf16_full_size():
     wl = synth.WORKLOADS["c3_etc_bf16"]
     q, k, v = synth.make_qkv(wl)
