@@ -755,12 +755,12 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                     const bool good = have && ((qbits >> r64) & 1ull) && l_sum > 0.f;
                     const size_t tok = ((size_t)slot->bh * p.nb + my_q) * kBlock + r64;
                     uint4* dst = reinterpret_cast<uint4*>(p.out + tok * kBlock);
-                    if (p.lse) p.lse[tok] = good ? (m_ref + log2f(l_sum)) * 0.6931471805599453f : -INFINITY;
+                    if (p.lse) p.lse[tok] = good ? (m_ref + __log2f(l_sum)) * 0.6931471805599453f : -INFINITY;
                     if (have) {
                         // the accumulator is read once the tile's last P V is known to be complete
                         pend_out = true;
                         pend_partial = false;
-                        pend_inv = good ? 1.f / l_sum : 0.f;
+                        pend_inv = good ? __frcp_rn(l_sum) : 0.f;
                         pend_dst = dst;
                     } else {
                         const uint4 z = make_uint4(0u, 0u, 0u, 0u);
