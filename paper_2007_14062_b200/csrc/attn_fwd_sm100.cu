@@ -331,7 +331,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         mbar_init(&ctl->s_free, kSoftmaxWarps * 32);    // every softmax thread arrives itself: cheaper than
         mbar_init(&ctl->p_full, kSoftmaxWarps * 32);    // converging the warp and electing a lane
         mbar_init(&ctl->pv_done, 1);
-        for (int i = 0; i < kSchedSlots; ++i) { mbar_init(&ctl->sched_full[i], 1); mbar_init(&ctl->sched_empty[i], 2 + kSoftmaxWarps); }
+        for (int i = 0; i < kSchedSlots; ++i) { mbar_init(&ctl->sched_full[i], 1); mbar_init(&ctl->sched_empty[i], 2 + kSoftmaxWarps * 32); }
         ctl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -770,8 +770,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                 }
             }
             tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&ctl->sched_empty[ss]);
+            mbar_arrive(&ctl->sched_empty[ss]);
             ++sched_n;
         }
     }
