@@ -60,7 +60,8 @@ typedef struct bigbird_layout bigbird_layout;   /* opaque */
  *   r     random key blocks per (head, non-global query block) (App. D item 1), drawn without replacement
  *         from the ascending list of blocks that are neither in the query block's window nor global (all of
  *         them if fewer than r).  The same for every batch element; not symmetrised (the graph is directed).
- *   seed  selects the random blocks.  The paper fixes no generator; this library's is: a SplitMix64 stream
+ *   seed  selects the random blocks; seed < 2^24, else BIGBIRD_EINVAL (the stream key below gives it 24 bits).
+ *         The paper fixes no generator; this library's is: a SplitMix64 stream
  *         with initial state (seed << 40) ^ (h << 20) ^ j for head h and query block j (h, j < 2^20), the
  *         bounded draw floor(z * m / 2^64), and a partial Fisher-Yates shuffle of the candidate list
  *         (for t < r: swap entries t and t + draw(m - t)); the first r entries are taken.
@@ -118,7 +119,8 @@ BIGBIRD_API int bigbird_layout_destroy(bigbird_layout* layout);
  * The first call on a device (and the first call with a larger B, N or a new layout) allocates device
  * scratch owned by the library; later calls allocate nothing.  That scratch (packed mask bits, partial results
  * of split global tiles) is per device: calls that use a key-padding mask or a layout with N/b > 96 must not
- * overlap on the GPU with other such calls (put them on one stream).
+ * overlap on the GPU with other such calls (put them on one stream).  Host threads may call concurrently: the
+ * library serialises its own bookkeeping.
  * Errors: BIGBIRD_EINVAL, BIGBIRD_EUNSUPPORTED, BIGBIRD_ECUDA, BIGBIRD_ENOMEM.  There is no CPU path.
  */
 BIGBIRD_API int bigbird_attn_fwd(const void* q, const void* k, const void* v, const bigbird_layout* layout,
@@ -152,16 +154,19 @@ BIGBIRD_API int bigbird_attn_fwd_simt(const void* q, const void* k, const void* 
  *     steps summed over heads (bigbird_layout_schedule reports both), and N/b <= 96 (longer sequences have
  *     their global tiles split into parts whose partial results need scratch that grows with B * H); beyond
  *     them the call does nothing and returns BIGBIRD_ELIMIT;
- *   - the schedule of `layout` is copied from host to device on every call (two cudaMemcpyAsync on `stream`),
- *     so `layout` must not be destroyed while the call is being enqueued;
+ *   - the array holds the device copy of one layout's schedule.  A call with another layout than the previous
+ *     call on that device first copies the new schedule from the handle's host arrays (two cudaMemcpyAsync on
+ *     `stream` from pageable memory: the host may wait until they have been staged); later calls with the same
+ *     layout enqueue only a 16-byte cudaMemsetAsync and the kernels.  `layout` must not be destroyed while a
+ *     call that uses it is being enqueued;
  *   - the first call on a device looks up the array's device address and sets a kernel attribute; make that
  *     first call outside any stream capture;
  *   - all calls on a device share the array, which keeps the contents of the last call: the entry point
  *     re-initialises what must start at zero, but two calls whose kernels overlap on the GPU (different
  *     streams, or different threads) race on it and give undefined results.  Serialise them;
- *   - a bounded wait that expires inside the kernel is not reported by bigbird_last_status (that function reads
- *     the allocated scratch of bigbird_attn_fwd), and bigbird_last_launch_count / bigbird_last_cuda_error are
- *     not updated.
+ *   - a bounded wait that expires inside the kernel is reported by bigbird_last_status_static, not by
+ *     bigbird_last_status (which reads the allocated scratch of bigbird_attn_fwd); bigbird_last_launch_count and
+ *     bigbird_last_cuda_error are not updated.
  * Errors: BIGBIRD_EINVAL, BIGBIRD_EUNSUPPORTED, BIGBIRD_ELIMIT, BIGBIRD_ECUDA.
  */
 BIGBIRD_API int bigbird_attn_fwd_static(const void* q, const void* k, const void* v, const bigbird_layout* layout,
@@ -169,9 +174,21 @@ BIGBIRD_API int bigbird_attn_fwd_static(const void* q, const void* k, const void
                             int B, int H, int64_t N, int D, int b, float scale, int dtype, void* stream);
 
 /*
+ * bigbird_last_status_static -- the status of the last bigbird_attn_fwd_static call on the current device:
+ * synchronises `stream`, then reads the two status words at the head of the fixed array into a host stack buffer
+ * (no allocation).  *status is BIGBIRD_OK or BIGBIRD_ETIMEOUT, *detail (may be NULL) names the wait.  Every
+ * bigbird_attn_fwd_static call clears the words when it starts.
+ */
+BIGBIRD_API int bigbird_last_status_static(void* stream, int* status, int* detail);
+
+/*
  * bigbird_last_status -- synchronises `stream` and reads the device status word of the current device:
  * BIGBIRD_OK, or BIGBIRD_ETIMEOUT if a bounded wait inside a kernel gave up (the kernel then returned early and
  * its outputs are invalid).  *detail (may be NULL) receives a code naming the wait.  Clears the word.
+ * The word is one per device, shared by every bigbird_attn_fwd launch on it, so a timeout cannot be attributed to
+ * one call among several in flight; after a timeout the function also resets the work counters of every launch
+ * slot on that device (with a blocking cudaMemset), which is only safe once all attention kernels on the device
+ * have finished.  A debugging facility: call it with the device otherwise idle.
  */
 BIGBIRD_API int bigbird_last_status(void* stream, int* status, int* detail);
 

@@ -33,9 +33,10 @@ Readings taken where the paper is silent (each is a deliberate choice):
   (Steele, Lea, Flood 2014; Vigna's public-domain constants) whose initial
   state is (seed << 40) ^ (h << 20) ^ j, a bounded draw floor(z * m / 2^64),
   and a partial Fisher-Yates shuffle of the candidate list.
-  PARITY UNPINNED by the paper for the random choice itself: the paper prints
-  no sample layout.  The stream is pinned to SplitMix64's published outputs,
-  and the selection to its invariants and statistics.
+  The paper prints no sample layout; the stream is pinned to SplitMix64's
+  published outputs and the selection to vectors worked by hand from them
+  (tests/golden/random_blocks_seed0.txt), besides its invariants and statistics.
+  seed < 2^24 and h, j < 2^20 (the key's field widths).
 * Padding: keys whose key_padding_mask is 0 get score -inf before the softmax;
   the attention graph itself does not depend on the mask.
 * lse is the natural log of the sum of exp(scaled, masked scores).
@@ -75,6 +76,9 @@ class Graph:
             raise ValueError("bad g, r or H")
         if self.mode not in (ITC, ETC):
             raise ValueError("mode")
+        # field widths of the stream key (seed << 40) ^ (h << 20) ^ j: 24 bits of seed, 20 of head, 20 of block
+        if not (0 <= self.seed < (1 << 24)) or self.H > (1 << 20) or self.N // self.b > (1 << 20):
+            raise ValueError("seed must be below 2^24, heads and blocks at most 2^20")
 
     @property
     def nb(self) -> int:

@@ -19,6 +19,7 @@ from .binding import (  # noqa: F401
     bigbird_build_layout,
     bigbird_last_launch_count,
     bigbird_last_status,
+    bigbird_last_status_static,
     bigbird_selftest_wait_expiry,
     bigbird_strerror,
     lib,

@@ -51,13 +51,14 @@ def lib() -> C.CDLL:
     L.bigbird_attn_fwd_simt.argtypes = fwd
     L.bigbird_attn_fwd_static.argtypes = fwd
     L.bigbird_last_status.argtypes = [vp, C.POINTER(i32), C.POINTER(i32)]
+    L.bigbird_last_status_static.argtypes = [vp, C.POINTER(i32), C.POINTER(i32)]
     L.bigbird_last_cuda_error.argtypes = []
     L.bigbird_selftest_wait_expiry.argtypes = [vp]
     L.bigbird_last_launch_count.argtypes = []
     L.bigbird_strerror.argtypes = [i32]
     L.bigbird_strerror.restype = C.c_char_p
     for name in ("bigbird_build_layout", "bigbird_layout_nnz", "bigbird_layout_export", "bigbird_layout_schedule",
-                 "bigbird_layout_destroy", "bigbird_attn_fwd", "bigbird_attn_fwd_simt", "bigbird_attn_fwd_static", "bigbird_last_status",
+                 "bigbird_layout_destroy", "bigbird_attn_fwd", "bigbird_attn_fwd_simt", "bigbird_attn_fwd_static", "bigbird_last_status", "bigbird_last_status_static",
                  "bigbird_last_cuda_error", "bigbird_last_launch_count", "bigbird_selftest_wait_expiry"):
         getattr(L, name).restype = i32
     _lib = L
@@ -170,6 +171,15 @@ def bigbird_last_status(stream: Optional[int] = None) -> Tuple[int, int]:
     if stream is None:
         stream = torch.cuda.current_stream().cuda_stream
     _check(lib().bigbird_last_status(C.c_void_p(stream), C.byref(st), C.byref(det)), "bigbird_last_status")
+    return st.value, det.value
+
+
+def bigbird_last_status_static(stream: Optional[int] = None) -> Tuple[int, int]:
+    """(status, detail) of the last bigbird_attn_fwd_static call on the current device; allocates nothing."""
+    st, det = C.c_int(0), C.c_int(0)
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    _check(lib().bigbird_last_status_static(C.c_void_p(stream), C.byref(st), C.byref(det)), "bigbird_last_status_static")
     return st.value, det.value
 
 

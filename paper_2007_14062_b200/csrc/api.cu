@@ -69,13 +69,9 @@ int get_device_layout(const bigbird_layout* L, int device, DeviceLayout* out) {
             free_device_layout(d);
             cudaSetDevice(cur);
         }
-        // steps are stored per head with head-relative item offsets: make item offsets absolute on upload
-        std::vector<Item> items = L->items;
-        for (int h = 0; h < L->H; ++h)
-            for (int i = 0; i < L->items_per_head; ++i) items[(size_t)h * L->items_per_head + i].step_begin += L->step_base[h];
         cudaError_t e = upload(&d.row_ptr, L->row_ptr.data(), L->row_ptr.size());
         if (e == cudaSuccess) e = upload(&d.col_idx, L->col_idx.data(), L->col_idx.size());
-        if (e == cudaSuccess) e = upload(&d.items, items.data(), items.size());
+        if (e == cudaSuccess) e = upload(&d.items, L->items_abs.data(), L->items_abs.size());
         if (e == cudaSuccess) e = upload(&d.steps, L->steps.data(), L->steps.size());
         if (e == cudaSuccess) e = upload(&d.split_tile_q, L->split_tile_q.data(), L->split_tile_q.size());
         if (e != cudaSuccess) { free_device_layout(d); return cuda_fail(e); }

@@ -6,24 +6,29 @@
 //   * Two query blocks are stacked into one 128-row tile so that every tcgen05.mma runs at M = 128.  The tile
 //     walks a list of key blocks prepared on the host; each is attended by both halves of the tile or by one.
 //     The MMAs always cover all 128 rows; rows that do not attend a key block get probability zero for it.
+//   * One CTA per SM runs two independent tile streams side by side.  Each stream owns half of tensor memory
+//     (scores 128 | probabilities 64 | output accumulator 64 columns), a Q double buffer and a ring of K / V
+//     tiles in shared memory, an MMA-issuing thread and a softmax warpgroup.  Two issuing threads keep the
+//     tensor pipe full where one thread's issue rate would not (a 64-wide P V instruction takes the pipe less
+//     time than one thread needs to issue the next), and the two softmax warpgroups fill each other's gaps on
+//     the special-function unit.
 //   * A producer thread fetches Q once per tile and the K and V blocks with TMA (128-byte swizzle) straight
-//     from the [B, H, N, D] tensors into a shared-memory ring: nothing is gathered or packed in HBM.
+//     from the [B, H, N, D] tensors into the stream's ring: nothing is gathered or packed in HBM.
 //   * Key blocks are processed two at a time (one "step").  Their K tiles land in adjacent ring slots, so that
-//     S = Q K^T of a step is one N = 128 tcgen05.mma per 16 head dimensions (an MMA instruction costs its issuing
-//     thread about the same time whatever its N, so wide MMAs are the cheap ones).  O += P V follows with P read
+//     S = Q K^T of a step is one N = 128 tcgen05.mma per 16 head dimensions.  O += P V follows with P read
 //     from tensor memory.
-//   * Four softmax warps, one thread per row of the tile: the thread pulls its (up to) 128 scores into registers
+//   * Softmax warpgroup, one thread per row of the tile: the thread pulls its (up to) 128 scores into registers
 //     with tcgen05.ld and hands the score columns back at once, so that the next step's Q K^T runs under this
 //     step's exponentials; it applies the key-padding mask, takes the row maximum, exponentiates (base 2, fp32),
 //     sums, and writes bf16 probabilities with tcgen05.st (zeros for key blocks its half of the tile does not
-//     attend); the previous step's P V runs under the first half of that.  The accumulator is rescaled only
-//     when the running maximum grows by more than 2^8.  The output of a tile is written during the first step
-//     of the next tile.
+//     attend).  The accumulator is rescaled only when the running maximum grows by more than 2^8.
+//   * An epilogue warpgroup shared by the two streams takes a finished tile's accumulator out of tensor memory,
+//     scales it by 1/l and writes the output rows, while the stream's softmax threads are already on the next tile.
 //   * A global-row tile of a long sequence is cut along the keys into parts that are separate work items; each
 //     writes its unnormalised accumulator and (max, sum) per row to scratch, and a small merge kernel combines
 //     the parts in a fixed order.
-//   * CTAs are persistent and draw work from a global counter: global-row tiles first, then the sparse tiles
-//     in (batch, head)-major order.  Two CTAs share an SM so that one's softmax overlaps the other's MMAs.
+//   * CTAs are persistent; a scheduler warp draws work for both streams from a global counter: global-row tiles
+//     first, then the sparse tiles in (batch, head)-major order.
 //
 // Every wait on an mbarrier is bounded: on expiry the kernel records BIGBIRD_ETIMEOUT and returns.
 #include <cuda.h>
@@ -45,15 +50,23 @@ constexpr int kTileBytes = kBlock * kBlock * 2;      // one 64x64 bf16 tile
 constexpr int kStepChunks = 2;             // key blocks per step
 constexpr int kRingGroups = 4;             // ring of groups of kStepChunks adjacent tiles (the K or the V blocks of one step)
 constexpr int kGroupBytes = kStepChunks * kTileBytes;
-constexpr int kThreads = 256;              // warp 0 TMA, warp 1 MMA issuer, warp 2 scheduler, warp 3 idle, warps 4..7 softmax
-constexpr int kSoftmaxWarps = 4;
-#ifndef BB_REGS_LIGHT
-#define BB_REGS_LIGHT 72
+constexpr int kStreams = 2;                // tile streams per CTA
+// warps 0..3 / 4..7: softmax of stream 0 / 1; warps 8..11: epilogue; warp 12: TMA producer; warps 13, 14: MMA issuers
+// of stream 0 / 1; warp 15: scheduler
+constexpr int kThreads = 512;
+constexpr int kWarpEpilogue = 8, kWarpProducer = 12, kWarpMma = 13, kWarpScheduler = 15;
+constexpr int kSoftmaxThreads = 128;
+#ifndef BB_REGS_SOFTMAX
 #define BB_REGS_SOFTMAX 184
+#define BB_REGS_EPILOGUE 80
+#define BB_REGS_LIGHT 64
 #endif
-constexpr int kRegsLight = BB_REGS_LIGHT;             // registers per thread of warps 0..3 after setmaxnreg
-constexpr int kRegsSoftmax = BB_REGS_SOFTMAX;          // registers per thread of warps 4..7 after setmaxnreg
-constexpr int kTmemCols = 256;
+constexpr int kRegsSoftmax = BB_REGS_SOFTMAX;          // registers per thread after setmaxnreg, by role
+constexpr int kRegsEpilogue = BB_REGS_EPILOGUE;
+constexpr int kRegsLight = BB_REGS_LIGHT;
+static_assert(kStreams * kRegsSoftmax + kRegsEpilogue + kRegsLight <= 512, "register file: 65536 = 128 threads x 512");
+constexpr int kTmemCols = 512;
+constexpr int kStreamCols = kTmemCols / kStreams;
 constexpr int kColS = 0;                   // scores: kStepChunks x 64 fp32 columns
 constexpr int kColP = kStepChunks * 64;    // probabilities: kStepChunks x 32 columns of packed bf16 pairs
 constexpr int kColO = kColP + kStepChunks * 32;   // output accumulator: 64 fp32 columns
@@ -62,7 +75,7 @@ constexpr long long kWaitLimitCycles = 4000000000ll;   // about two seconds
 constexpr int kSchedSlots = 3;
 constexpr int kPartialFloats = 128 * 64 + 2 * 128;   // one part of a split tile: O[128][64], max[128], sum[128]
 constexpr int kSegChunks = 96;             // live key blocks per posted segment of a tile (a multiple of kStepChunks)
-static_assert(kColO + 64 <= kTmemCols && kSegChunks % kStepChunks == 0, "tensor-memory and segment layout");
+static_assert(kColO + 64 <= kStreamCols && kSegChunks % kStepChunks == 0, "tensor-memory and segment layout");
 
 // A key block of a tile after the key-padding mask has been applied.
 struct __align__(16) ChunkEntry {
@@ -82,21 +95,39 @@ struct __align__(16) WorkSlot {
     unsigned long long qbits_a, qbits_b;
     ChunkEntry chunks[kSegChunks];         // step s of the segment covers chunks [kStepChunks s, kStepChunks (s + 1))
 };
+// What the softmax threads of a stream hand to the epilogue warpgroup at the end of a tile.
+enum { kEpiTile = 0, kEpiDone = 1 };
+struct __align__(16) EpiMsg {
+    int kind;                      // kEpiTile, or kEpiDone: the stream has no more tiles
+    int bh, qa, qb;
+    int part_slot;
+    int pad_[3];
+    float inv[kSoftmaxThreads];    // per row: 1 / l, or 0 for a row that must come out as zeros
+};
 
-struct __align__(16) SmemCtl {
+struct __align__(16) StreamCtl {
     unsigned long long full[kRingGroups];
     unsigned long long empty[kRingGroups];
     unsigned long long q_full[2], q_empty[2];
     unsigned long long s_full, s_free, p_full, pv_done;
+    unsigned long long o_done, o_free;     // a tile's last P V has completed / the epilogue has taken the accumulator
+    unsigned long long epi_full[2];
     unsigned long long sched_full[kSchedSlots], sched_empty[kSchedSlots];
+    WorkSlot slot[kSchedSlots];
+    EpiMsg epi[2];
+};
+struct __align__(16) SmemCtl {
+    StreamCtl st[kStreams];
     unsigned tmem_base;
     int abort_flag;
-    WorkSlot slot[kSchedSlots];
 };
-constexpr int kSmemQ = 0;
-constexpr int kSmemRing = 4 * kTileBytes;              // two Q buffers of two tiles each come first
-constexpr int kSmemCtl = kSmemRing + kRingGroups * kGroupBytes;
+// per stream: two Q buffers of two tiles each, then the ring
+constexpr int kStreamSmemQ = 0;
+constexpr int kStreamSmemRing = 4 * kTileBytes;
+constexpr int kStreamSmemBytes = kStreamSmemRing + kRingGroups * kGroupBytes;
+constexpr int kSmemCtl = kStreams * kStreamSmemBytes;
 constexpr int kSmemBytes = kSmemCtl + (int)sizeof(SmemCtl) + 1024;   // + slack for the 1024-byte alignment
+static_assert(kSmemBytes <= 227 * 1024, "shared memory per CTA");
 
 struct KernelParams {
     __nv_bfloat16* out;
@@ -141,29 +172,74 @@ __device__ __forceinline__ unsigned long long global_ns() {
     return t;
 }
 
+// One try with a limit on the time the thread stays suspended (nanoseconds): what a role that watches several
+// barriers sleeps on between rounds, so that it neither spins nor oversleeps the one it is suspended on.
+__device__ __forceinline__ bool mbar_try_for(unsigned long long* bar, unsigned parity, unsigned ns) {
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(ns) : "memory");
+    return ok != 0;
+}
+// Non-blocking test of a phase (for the roles that poll several barriers).
+__device__ __forceinline__ bool mbar_test(unsigned long long* bar, unsigned parity) {
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+
 // Bounded wait.  Returns false if the wait expired or another thread of the CTA already gave up.  The limit is
 // counted in SM clock cycles (a read of the cycle counter is cheap, unlike one of the global nanosecond timer)
 // and the counter is first read only after 64 failed tries.
-__device__ __forceinline__ bool mbar_wait_slow(unsigned long long* bar, unsigned parity, SmemCtl* ctl, int* status, int code) {
+__device__ __forceinline__ bool mbar_wait_slow(unsigned long long* bar, unsigned parity, int* abort_flag, int* status, int code) {
     long long t0 = 0;
     for (unsigned it = 0;; ++it) {
         if (mbar_try(bar, parity)) return true;
         if ((it & 63u) == 63u) {
-            if (*(volatile int*)&ctl->abort_flag) return false;
+            if (*(volatile int*)abort_flag) return false;
             const long long now = clock64();
             if (it == 63u) t0 = now;
             if (now - t0 > kWaitLimitCycles) {
                 if (atomicCAS(status, 0, BIGBIRD_ETIMEOUT) == 0) status[1] = code;
-                *(volatile int*)&ctl->abort_flag = 1;
+                *(volatile int*)abort_flag = 1;
                 return false;
             }
         }
     }
 }
-__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned parity, SmemCtl* ctl, int* status, int code) {
+__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned parity, int* abort_flag, int* status, int code) {
     if (__builtin_expect(mbar_try(bar, parity), 1)) return true;
-    return mbar_wait_slow(bar, parity, ctl, status, code);
+    return mbar_wait_slow(bar, parity, abort_flag, status, code);
 }
+// The same bound for a role that polls: tick() is called whenever a round over the role's barriers found nothing
+// to do; it backs off (a polling warp that spins takes issue slots from the softmax warps of its sub-partition)
+// and returns false once the CTA has given up or the idle time exceeds the limit.
+struct IdleClock {
+    unsigned n = 0;
+    long long t0 = 0;
+    __device__ __forceinline__ void reset() { n = 0; }
+    __device__ __forceinline__ bool tick(int* abort_flag, int* status, int code, unsigned sleep_ns) {
+        ++n;
+        if ((n & 15u) == 0u) {
+            if (*(volatile int*)abort_flag) return false;
+            const long long now = clock64();
+            if (n == 16u) t0 = now;
+            else if (now - t0 > kWaitLimitCycles) {
+                if (atomicCAS(status, 0, BIGBIRD_ETIMEOUT) == 0) status[1] = code;
+                *(volatile int*)abort_flag = 1;
+                return false;
+            }
+        }
+        if (sleep_ns) __nanosleep(sleep_ns);
+        return true;
+    }
+};
 
 __device__ __forceinline__ void tma_load_tile(void* dst, const CUtensorMap* tm, int row, unsigned long long* bar) {
     asm volatile(
@@ -298,7 +374,7 @@ __device__ __forceinline__ void fmul2(float& r0, float& r1, float a) {
         : "+f"(r0), "+f"(r1) : "f"(a));
 }
 
-// ------------------------------------------------------------------------------------------------ schedule helpers
+// ------------------------------------------------------------------------------------------------ helpers
 __device__ __forceinline__ unsigned long long key_bits(const KernelParams& p, int batch, int c) {
     if (c < 0) return 0ull;
     return p.kbits ? p.kbits[(size_t)batch * p.nb + c] : ~0ull;
@@ -315,8 +391,613 @@ __device__ __forceinline__ float row_max64(const float* s) {
     return fmaxf(max3(mx0, mx1, fmaxf(s[60], s[61])), max3(mx2, mx3, fmaxf(s[62], s[63])));
 }
 
+// Rare paths of the softmax threads.
+// -inf over the scores of the padded keys of one key block, in tensor memory.
+__device__ __forceinline__ void mask_scores(unsigned taddr, unsigned long long kb) {
+    float s[64];
+    tmem_ld64(taddr, s);
+    tmem_wait_ld();
+#pragma unroll
+    for (int t = 0; t < 64; ++t) s[t] = ((kb >> t) & 1ull) ? s[t] : -INFINITY;
+    tmem_st32(taddr, reinterpret_cast<unsigned*>(s));
+    tmem_st32(taddr + 32, reinterpret_cast<unsigned*>(s + 32));
+    tmem_wait_st();
+}
+// This thread's row of the output accumulator times alpha (the running maximum moved by more than the threshold).
+__device__ __forceinline__ void rescale_accumulator(unsigned taddr, float alpha) {
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        float o[16];
+        tmem_ld16(taddr + c * 16, o);
+        tmem_wait_ld();
+#pragma unroll
+        for (int t = 0; t < 16; t += 2) fmul2(o[t], o[t + 1], alpha);
+        tmem_st16(taddr + c * 16, reinterpret_cast<unsigned*>(o));
+    }
+}
+
+// What every role needs to know about its stream.
+struct StreamRef {
+    StreamCtl* sc;
+    unsigned char* smem;           // the stream's Q buffers and ring
+    unsigned tmem;                 // tensor-memory address of the stream's first column (lane 0)
+};
+
+// ------------------------------------------------------------------------------------------------ scheduler (one warp, both streams)
+// Fetches the next work item for a stream, drops the key blocks that are entirely padding and posts the live
+// list.  Returns the work index (-1: the stream has been told that there is no more work), or -2 after an
+// expired wait.
+__device__ __forceinline__ int schedule_one(const KernelParams& p, SmemCtl* ctl, StreamCtl* sc, unsigned& sched_n, int lane) {
+    const unsigned lt_mask = (1u << lane) - 1u;
+    int w = 0;
+    if (lane == 0) w = atomicAdd(&p.counter[0], 1);
+    w = __shfl_sync(0xffffffffu, w, 0);
+    if (w >= p.total_work) w = -1;
+    // decode the work index: global-row tiles of every (batch, head) first, then the sparse tiles
+    int bh = 0, it = 0;
+    Item item{};
+    if (w >= 0) {
+        const int heavy_total = p.BH * p.heavy_per_head;
+        if (w < heavy_total) {
+            bh = w / p.heavy_per_head;
+            it = w - bh * p.heavy_per_head;
+        } else {
+            const int sparse = p.items_per_head - p.heavy_per_head;
+            const int w2 = w - heavy_total;
+            bh = w2 / sparse;
+            it = p.heavy_per_head + (w2 - bh * sparse);
+        }
+        item = p.items[(size_t)(bh % p.H) * p.items_per_head + it];
+    }
+    const int batch = bh / p.H;
+    const unsigned long long qbits_a = w >= 0 ? key_bits(p, batch, item.qa) : 0ull;
+    const unsigned long long qbits_b = w >= 0 ? key_bits(p, batch, item.qb) : 0ull;
+    const bool tile_live = (qbits_a | qbits_b) != 0ull;      // a tile whose query rows are all padding is skipped
+    const int n_raw = (w >= 0 && tile_live) ? item.step_count : 0;
+    int i0 = 0;
+    bool first = true;
+    do {
+        const unsigned ss = sched_n % kSchedSlots, sp = (sched_n / kSchedSlots) & 1u;
+        // the first slot of an item is known to be free (the caller tested it); later segments of a long tile wait here
+        if (!mbar_wait(&sc->sched_empty[ss], sp ^ 1u, &ctl->abort_flag, p.status, 11)) return -2;
+        WorkSlot* slot = &sc->slot[ss];
+        int count = 0;
+        while (i0 < n_raw && count <= kSegChunks - 32) {
+            const int i = i0 + lane;
+            ChunkEntry e{-1, 0, 0ull};
+            bool alive = false;
+            if (i < n_raw) {
+                const Step s = p.steps[item.step_begin + i];
+                // halves whose query rows are all padding do not attend anything
+                const bool ua = s.who != kLowerHalf && qbits_a != 0ull;
+                const bool ub = s.who != kUpperHalf && qbits_b != 0ull;
+                e.c = s.c;
+                e.kb = key_bits(p, batch, s.c);
+                e.who = ((ua && ub) ? kBothHalves : (ua ? kUpperHalf : kLowerHalf)) | (e.kb != ~0ull ? kHasPadding : 0);
+                alive = e.kb != 0ull && (ua || ub);
+#ifdef BB_DEBUG
+                if (s.c < 0 || s.c >= p.nb) { debug_fail(ctl, p.status, 70); alive = false; }
+#endif
+            }
+            const unsigned bal = __ballot_sync(0xffffffffu, alive);
+            if (alive) slot->chunks[count + __popc(bal & lt_mask)] = e;
+            count += __popc(bal);
+            i0 += 32;
+        }
+        if (lane == 0) {
+            slot->w = w;
+            slot->bh = bh;
+            slot->batch = batch;
+            slot->qa = item.qa;
+            slot->qb = item.qb;
+            slot->n_chunks = count;
+            slot->flags = (first ? kSegFirst : 0) | (i0 >= n_raw ? kSegLast : 0) | (tile_live ? kSegLive : 0);
+            slot->qbits_a = qbits_a;
+            slot->qbits_b = qbits_b;
+            slot->part_slot = (w >= 0 && item.nparts > 1) ? ((bh * p.split_tiles_per_head + item.tile) * p.max_parts + item.part) : -1;
+        }
+        __threadfence_block();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sc->sched_full[ss]);
+        ++sched_n;
+        first = false;
+    } while (i0 < n_raw);
+    return w;
+}
+
+__device__ __forceinline__ void scheduler_role(const KernelParams& p, SmemCtl* ctl, int lane) {
+    unsigned sched_n[kStreams] = {0, 0};
+    unsigned done = 0;                              // bit s: stream s has been told that there is no more work
+    IdleClock idle;
+    while (done != (1u << kStreams) - 1u) {
+        bool progress = false;
+#pragma unroll 1
+        for (int s = 0; s < kStreams; ++s) {        // (not unrolled: one copy of the code)
+            if ((done >> s) & 1u) continue;
+            StreamCtl* sc = &ctl->st[s];
+            const unsigned ss = sched_n[s] % kSchedSlots, sp = (sched_n[s] / kSchedSlots) & 1u;
+            if (!__all_sync(0xffffffffu, mbar_test(&sc->sched_empty[ss], sp ^ 1u))) continue;
+            unsigned n = sched_n[s];
+            const int w = schedule_one(p, ctl, sc, n, lane);
+            sched_n[s] = n;
+            if (w == -2) return;
+            if (w < 0) done |= 1u << s;
+            progress = true;
+        }
+        if (progress) idle.reset();
+        else if (!__all_sync(0xffffffffu, idle.tick(&ctl->abort_flag, p.status, 12, 400))) return;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------ TMA producer (one thread per stream)
+// Ring order of a stream = the order in which its MMA thread consumes groups: K of step i, then V of step i-1.
+struct ProducerState {
+    unsigned ring_n = 0, q_n = 0, sched_n = 0;
+    int op = 0;                    // what the stream needs next (kOp*)
+    int w = 0, bh = 0, n = 0, i = 0;
+    int cur_n = 0, cur_c0 = 0, cur_c1 = 0;
+    int pend_n = 0, pend_bh = 0, pend_c0 = 0, pend_c1 = 0;
+};
+enum { kOpSlot = 0, kOpQ, kOpK, kOpV, kOpRelease, kOpFinalV, kOpDone };
+
+__device__ __forceinline__ void load_group(const KernelParams& p, const StreamRef& sr, const CUtensorMap* tm, unsigned g, int bh, int c0, int c1, int cnt) {
+    StreamCtl* sc = sr.sc;
+    mbar_expect_tx(&sc->full[g], cnt * kTileBytes);
+    tma_load_tile(sr.smem + kStreamSmemRing + g * kGroupBytes, tm, (bh * p.nb + c0) * kBlock, &sc->full[g]);
+    if (cnt > 1) tma_load_tile(sr.smem + kStreamSmemRing + g * kGroupBytes + kTileBytes, tm, (bh * p.nb + c1) * kBlock, &sc->full[g]);
+}
+
+// One non-blocking attempt to move the stream's loads forward.  Returns whether anything was done.
+__device__ __forceinline__ bool producer_advance(const KernelParams& p, const StreamRef& sr, ProducerState& st, const CUtensorMap* tm_q,
+                                                 const CUtensorMap* tm_k, const CUtensorMap* tm_v) {
+    StreamCtl* sc = sr.sc;
+    const unsigned ss = st.sched_n % kSchedSlots, sp = (st.sched_n / kSchedSlots) & 1u;
+    const WorkSlot* slot = &sc->slot[ss];
+    const unsigned g = st.ring_n % kRingGroups, gph = (st.ring_n / kRingGroups) & 1u;
+    switch (st.op) {
+        case kOpSlot: {
+            if (!mbar_test(&sc->sched_full[ss], sp)) return false;
+            st.w = slot->w;
+            st.bh = slot->bh;
+            st.n = slot->n_chunks;
+            st.i = 0;
+            const int flags = slot->flags;
+            if (st.w >= 0 && (flags & kSegLive)) st.op = (flags & kSegFirst) ? kOpQ : (st.n > 0 ? kOpK : kOpRelease);
+            else st.op = kOpRelease;
+            return true;
+        }
+        case kOpQ: {
+            const unsigned qs = st.q_n & 1u;
+            if (!mbar_test(&sc->q_empty[qs], ((st.q_n >> 1) & 1u) ^ 1u)) return false;
+            const int qa = slot->qa, qb = slot->qb;
+            mbar_expect_tx(&sc->q_full[qs], qb >= 0 ? 2 * kTileBytes : kTileBytes);
+            tma_load_tile(sr.smem + kStreamSmemQ + qs * 2 * kTileBytes, tm_q, (st.bh * p.nb + qa) * kBlock, &sc->q_full[qs]);
+            if (qb >= 0) tma_load_tile(sr.smem + kStreamSmemQ + qs * 2 * kTileBytes + kTileBytes, tm_q, (st.bh * p.nb + qb) * kBlock, &sc->q_full[qs]);
+            ++st.q_n;
+            st.op = st.n > 0 ? kOpK : kOpRelease;
+            return true;
+        }
+        case kOpK: {
+            if (!mbar_test(&sc->empty[g], gph ^ 1u)) return false;
+            st.cur_n = min(kStepChunks, st.n - st.i);
+            st.cur_c0 = slot->chunks[st.i].c;
+            st.cur_c1 = st.cur_n > 1 ? slot->chunks[st.i + 1].c : 0;
+            load_group(p, sr, tm_k, g, st.bh, st.cur_c0, st.cur_c1, st.cur_n);
+            ++st.ring_n;
+            if (st.pend_n > 0) { st.op = kOpV; return true; }
+            break;                                          // no V pending: straight to the bookkeeping below
+        }
+        case kOpV: {
+            if (!mbar_test(&sc->empty[g], gph ^ 1u)) return false;
+            load_group(p, sr, tm_v, g, st.pend_bh, st.pend_c0, st.pend_c1, st.pend_n);
+            ++st.ring_n;
+            break;
+        }
+        case kOpRelease: {
+            mbar_arrive(&sc->sched_empty[ss]);
+            ++st.sched_n;
+            st.op = st.w < 0 ? (st.pend_n > 0 ? kOpFinalV : kOpDone) : kOpSlot;
+            return true;
+        }
+        case kOpFinalV: {
+            if (!mbar_test(&sc->empty[g], gph ^ 1u)) return false;
+            load_group(p, sr, tm_v, g, st.pend_bh, st.pend_c0, st.pend_c1, st.pend_n);
+            ++st.ring_n;
+            st.pend_n = 0;
+            st.op = kOpDone;
+            return true;
+        }
+        default: return false;
+    }
+    // the step's K (and the previous step's V) are on their way: this step's V becomes the pending one
+    st.pend_n = st.cur_n;
+    st.pend_bh = st.bh;
+    st.pend_c0 = st.cur_c0;
+    st.pend_c1 = st.cur_c1;
+    st.i += kStepChunks;
+    st.op = st.i < st.n ? kOpK : kOpRelease;
+    return true;
+}
+
+// Lane s of the producer warp serves stream s: the lanes run the same loop side by side, so that the two
+// streams' copies are issued by the same instructions most of the time.
+__device__ __forceinline__ void producer_role(const KernelParams& p, SmemCtl* ctl, const StreamRef& sr,
+                                              const CUtensorMap* tm_q, const CUtensorMap* tm_k, const CUtensorMap* tm_v) {
+    ProducerState st;
+    IdleClock idle;
+    while (st.op != kOpDone) {
+        if (producer_advance(p, sr, st, tm_q, tm_k, tm_v)) idle.reset();
+        else if (!idle.tick(&ctl->abort_flag, p.status, 10, 40)) return;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------ MMA issuer (one thread per stream)
+__device__ __forceinline__ void mma_role(const KernelParams& p, SmemCtl* ctl, const StreamRef& sr) {
+    StreamCtl* sc = sr.sc;
+    int* abort_flag = &ctl->abort_flag;
+    unsigned ring_n = 0, q_n = 0, sched_n = 0, grp_n = 0, pv_n = 0, tile_n = 0;   // grp_n: steps whose Q K^T was issued; tile_n: tiles handed to the epilogue
+    bool ok = true;
+    auto qk = [&](int cnt, unsigned qs) -> bool {   // S[:, 0 .. 64 cnt) = Q K^T with the K blocks of the next ring group
+        const unsigned g = ring_n % kRingGroups, ph = (ring_n / kRingGroups) & 1u;
+        if (!mbar_wait(&sc->full[g], ph, abort_flag, p.status, 20)) return false;
+        tc_fence_after();
+        // the blocks of a group are adjacent: their 64 cnt rows form one K-major operand
+        const unsigned long long q_desc = smem_desc_sw128(smem_u32(sr.smem + kStreamSmemQ + qs * 2 * kTileBytes));
+        const unsigned long long k_desc = smem_desc_sw128(smem_u32(sr.smem + kStreamSmemRing + g * kGroupBytes));
+        const unsigned idesc = kIdescQK64 + ((unsigned)(cnt - 1) << 20);           // N = 64 cnt
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)          // 16 head dims (32 bytes inside the swizzled row) per MMA
+            mma_ss(sr.tmem + kColS, q_desc + (unsigned long long)(kk * 2), k_desc + (unsigned long long)(kk * 2), idesc, kk > 0);
+        tc_commit(&sc->empty[g]);
+        ++ring_n;
+        return true;
+    };
+    bool pend_fresh = false;                    // the pending P V is the first of its tile: it overwrites O
+    bool pend_last = false;                     // ... the last of its tile: the accumulator is complete after it
+    bool tile_fresh = false, q_unseen = false;
+    int pend_n = 0, tile_steps = 0;
+    auto pending_pv = [&]() -> bool {           // O (+)= sum_j P_j V_j with the V blocks of the next ring group
+        if (pend_n == 0) return true;
+        if (!mbar_wait(&sc->p_full, pv_n & 1u, abort_flag, p.status, 22)) return false;
+        // the epilogue must have taken the previous tile's accumulator before this tile's first P V overwrites it
+        if (pend_fresh && tile_n > 0 && !mbar_wait(&sc->o_free, (tile_n - 1) & 1u, abort_flag, p.status, 27)) return false;
+        const unsigned g = ring_n % kRingGroups, ph = (ring_n / kRingGroups) & 1u;
+        if (!mbar_wait(&sc->full[g], ph, abort_flag, p.status, 21)) return false;
+        tc_fence_after();
+        const unsigned long long v_desc = smem_desc_sw128(smem_u32(sr.smem + kStreamSmemRing + g * kGroupBytes));
+#pragma unroll
+        for (int j = 0; j < kStepChunks; ++j) {
+            if (j < pend_n) {
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)  // 16 keys per MMA: 8 packed columns of P_j, two 8-row groups of V_j
+                    mma_ts(sr.tmem + kColO, sr.tmem + kColP + 32 * j + kk * 8, v_desc + (unsigned long long)((j * kTileBytes + kk * 2048) >> 4), kIdescPV,
+                           (j > 0 || kk > 0 || !pend_fresh) ? 1u : 0u);
+            }
+        }
+        tc_commit(&sc->empty[g]);
+        tc_commit(&sc->pv_done);
+        if (pend_last) {
+            tc_commit(&sc->o_done);
+            ++tile_n;
+        }
+        ++ring_n;
+        ++pv_n;
+        pend_n = 0;
+        pend_fresh = false;
+        pend_last = false;
+        return true;
+    };
+    while (ok) {
+        const unsigned ss = sched_n % kSchedSlots, sp = (sched_n / kSchedSlots) & 1u;
+        if (!mbar_wait(&sc->sched_full[ss], sp, abort_flag, p.status, 23)) break;
+        const WorkSlot* slot = &sc->slot[ss];
+        const int w = slot->w, flags = slot->flags, n = slot->n_chunks;
+        if (w >= 0 && (flags & kSegLive) && (flags & kSegFirst)) {
+            ++q_n;                              // this tile's Q sits in buffer (q_n - 1) & 1
+            q_unseen = true;
+            tile_fresh = true;
+            tile_steps = 0;
+        }
+        const bool work = w >= 0 && (flags & kSegLive);
+        const unsigned qs = (q_n - 1) & 1u, qph = ((q_n - 1) >> 1) & 1u;
+        // one round per step of the slot: this step's Q K^T, then the previous step's P V behind it; the slot that
+        // says "no more work" gets one round without a Q K^T, which issues the very last P V
+        const int n_rounds = work ? (n + kStepChunks - 1) / kStepChunks : (w < 0 ? 1 : 0);
+        for (int r = 0; r < n_rounds && ok; ++r) {
+            int cnt = 0;
+            if (work) {
+                // the softmax threads must have pulled the previous scores out of tensor memory
+                if (grp_n > 0) {
+                    ok = mbar_wait(&sc->s_free, (grp_n - 1) & 1u, abort_flag, p.status, 25);
+                    if (!ok) break;
+                }
+                if (q_unseen) {
+                    ok = mbar_wait(&sc->q_full[qs], qph, abort_flag, p.status, 24);
+                    if (!ok) break;
+                    q_unseen = false;
+                }
+                tc_fence_after();
+                cnt = min(kStepChunks, n - r * kStepChunks);
+                ok = qk(cnt, qs);
+                if (!ok) break;
+                tc_commit(&sc->s_full);
+                ++grp_n;
+            }
+            ok = pending_pv();
+            if (work) {
+                pend_n = cnt;
+                pend_fresh = tile_fresh;
+                tile_fresh = false;
+                ++tile_steps;
+            }
+        }
+        if (!ok) break;
+        if (work && (flags & kSegLast)) {
+            if (q_unseen) {                     // a tile without a live key block: its Q still has to land
+                ok = mbar_wait(&sc->q_full[qs], qph, abort_flag, p.status, 26);
+                if (!ok) break;
+                q_unseen = false;
+            }
+            tc_commit(&sc->q_empty[qs]);       // every Q K^T of the tile has been issued
+            if (tile_steps > 0) pend_last = true;           // the tile's last P V is the pending one
+        }
+        mbar_arrive(&sc->sched_empty[ss]);
+        ++sched_n;
+        if (w < 0) break;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------ softmax (one warpgroup per stream, one thread per row)
+__device__ __forceinline__ void softmax_role(const KernelParams& p, SmemCtl* ctl, const StreamRef& sr, int warp, int lane) {
+    StreamCtl* sc = sr.sc;
+    int* abort_flag = &ctl->abort_flag;
+    const int quad = warp & 3;                      // tensor-memory lanes this warp may touch: 32*quad .. +31
+    const int row = quad * 32 + lane;               // row of the 128-row tile
+    const bool lower = row >= kBlock;
+    const int my_who = lower ? kLowerHalf : kUpperHalf;
+    const unsigned lane_addr = sr.tmem + ((unsigned)(quad * 32) << 16);
+    const float sl2 = p.scale_log2;
+    unsigned sched_n = 0, grp_n = 0, msg_n = 0;
+    bool ok = true;
+    float m_ref = -INFINITY, l_sum = 0.f;
+    bool o_dirty = false;                           // has any P V been issued for this tile yet
+    // exponentials of the 64 scores of one key block, packed in place: afterwards s[0..31] hold the bit
+    // patterns of the 32 words of bf16 probability pairs
+    auto exp_pack = [&](float* s, float neg_m, float& sum0, float& sum1) {
+#pragma unroll
+        for (int t = 0; t < 64; t += 2) {
+            float t0, t1;
+            ffma2(t0, t1, s[t], s[t + 1], sl2, neg_m);
+            const float p0 = ex2(t0), p1 = ex2(t1);
+            fadd2(sum0, sum1, p0, p1);
+            s[t >> 1] = __uint_as_float(pack_bf16(p0, p1));
+        }
+    };
+    while (ok) {
+        const unsigned ss = sched_n % kSchedSlots, sp = (sched_n / kSchedSlots) & 1u;
+        if (!mbar_wait(&sc->sched_full[ss], sp, abort_flag, p.status, 30)) break;
+        __syncwarp();
+        const WorkSlot* slot = &sc->slot[ss];
+        const int w = slot->w, flags = slot->flags, n = slot->n_chunks;
+        if (w < 0) {                                // tell the epilogue that this stream is finished
+            // (once it has taken the last tile: only then is it known to have read every earlier message, so that
+            // the entry reused here is free)
+            if (msg_n > 0 && !mbar_wait(&sc->o_free, (msg_n - 1) & 1u, abort_flag, p.status, 36)) break;
+            EpiMsg* msg = &sc->epi[msg_n & 1u];
+            if (row == 0) msg->kind = kEpiDone;
+            mbar_arrive(&sc->epi_full[msg_n & 1u]);
+            break;
+        }
+        const bool live = flags & kSegLive;
+        if (flags & kSegFirst) {
+            m_ref = -INFINITY;
+            l_sum = 0.f;
+            o_dirty = false;
+        }
+        for (int i = 0; i < n && ok; i += kStepChunks) {
+            const ChunkEntry* e = &slot->chunks[i];
+            const int cnt = min(kStepChunks, n - i);
+            // which of the step's key blocks my half of the tile attends (warp-uniform)
+            const int who0 = e[0].who, who1 = cnt > 1 ? e[1].who : kNoChunk;
+            const bool mine0 = (who0 & kWhoMask) == kBothHalves || (who0 & kWhoMask) == my_who;
+            const bool mine1 = (who1 & kWhoMask) == kBothHalves || (who1 & kWhoMask) == my_who;
+            ok = mbar_wait(&sc->s_full, grp_n & 1u, abort_flag, p.status, 31);
+            if (!ok) break;
+            __syncwarp();                           // lanes leave the wait one by one: back in step before the warp-wide loads
+            tc_fence_after();
+            // A key block with padded keys (rare: the one holding a sequence's end) gets -inf written over their
+            // scores in tensor memory first, so that the common path below carries no masking code at all.
+            if (__builtin_expect(((who0 | who1) & kHasPadding) != 0, 0)) {
+                if (mine0 && (who0 & kHasPadding)) mask_scores(lane_addr + kColS, e[0].kb);
+                if (mine1 && (who1 & kHasPadding)) mask_scores(lane_addr + kColS + 64, e[1].kb);
+            }
+            // Two passes over the scores, each pulling them out of tensor memory: the row maximum first, then the
+            // exponentials one key block at a time in a loop that is not unrolled.  Reading twice is cheap; code that
+            // held all 128 scores in registers and was written out per key block was several times the size, and
+            // the kernel was bound by instruction fetch.
+            float alpha = 1.f;
+            bool rescale = false;
+            if (mine0 || mine1) {
+                float m_loc = -INFINITY;
+#pragma unroll 1
+                for (int c = 0; c < cnt; ++c) {
+                    if (!((c == 0 ? mine0 : mine1))) continue;
+                    float s[64];
+                    tmem_ld64(lane_addr + kColS + 64 * c, s);
+                    tmem_wait_ld();
+                    m_loc = fmaxf(m_loc, row_max64(s));
+                }
+                const float m_cand = m_loc * sl2;
+                const bool need = m_cand > m_ref + kRescaleThreshold;        // true on the first step (m_ref = -inf)
+                rescale = __any_sync(0xffffffffu, need);
+                if (need) {
+                    alpha = ex2(m_ref - m_cand);
+                    m_ref = m_cand;
+                }
+            } else {
+                // nothing of this step is mine: the score columns are free as far as this thread is concerned
+                tc_fence_before();
+                mbar_arrive(&sc->s_free);
+            }
+            float sum0 = 0.f, sum1 = 0.f;
+            const float neg_m = -m_ref;
+            const unsigned mine_bits = (mine0 ? 1u : 0u) | (mine1 ? 2u : 0u);
+#pragma unroll 1
+            for (int c = 0; c < cnt; ++c) {
+                const bool mine = (mine_bits >> c) & 1u;
+                float s[64];
+                if (mine) {
+                    tmem_ld64(lane_addr + kColS + 64 * c, s);
+                    tmem_wait_ld();
+                    if ((mine_bits >> (c + 1)) == 0u) {
+                        // my last scores of the step are in registers: the next step's Q K^T may overwrite the columns
+                        tc_fence_before();
+                        mbar_arrive(&sc->s_free);
+                    }
+                    exp_pack(s, neg_m, sum0, sum1);
+                }
+                if (c == 0) {
+                    // the previous step's P V must be complete before its probabilities are overwritten or O is touched
+                    if (grp_n > 0) {
+                        ok = mbar_wait(&sc->pv_done, (grp_n - 1) & 1u, abort_flag, p.status, 32);
+                        if (!ok) break;
+                        __syncwarp();
+                        tc_fence_after();
+                    }
+                    if (__builtin_expect(rescale && o_dirty, 0)) rescale_accumulator(lane_addr + kColO, alpha);
+                }
+                if (mine) tmem_st32(lane_addr + kColP + 32 * c, reinterpret_cast<unsigned*>(s));
+                else tmem_st32_zero(lane_addr + kColP + 32 * c);
+            }
+            if (!ok) break;
+            l_sum = l_sum * alpha + (sum0 + sum1);
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(&sc->p_full);
+            ++grp_n;
+            o_dirty = true;
+        }
+        if (!ok) break;
+        if (flags & kSegLast) {
+            // -------------------------------------------------------- end of the tile: lse now, the output rows via the epilogue
+            const int my_q = lower ? slot->qb : slot->qa;
+            const unsigned long long qbits = lower ? slot->qbits_b : slot->qbits_a;
+            const bool have = live && o_dirty;
+            const int part_slot = slot->part_slot;
+            const int r64 = row & (kBlock - 1);
+            float inv = 0.f;
+            if (part_slot >= 0) {
+                // one part of a split tile: (max, sum) from here, the raw accumulator from the epilogue
+                float* part = p.partials + (size_t)part_slot * kPartialFloats;
+                part[128 * 64 + row] = have ? m_ref : -INFINITY;
+                part[128 * 64 + 128 + row] = have ? l_sum : 0.f;
+            } else if (my_q >= 0) {                 // warp-uniform
+                const bool good = have && ((qbits >> r64) & 1ull) && l_sum > 0.f;
+                const size_t tok = ((size_t)slot->bh * p.nb + my_q) * kBlock + r64;
+                if (p.lse) p.lse[tok] = good ? (m_ref + __log2f(l_sum)) * 0.6931471805599453f : -INFINITY;
+                inv = good ? __frcp_rn(l_sum) : 0.f;
+                if (!have) {                        // no key block was attended: the row is zeros, written from here
+                    uint4* dst = reinterpret_cast<uint4*>(p.out + tok * kBlock);
+                    const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) dst[j] = z;
+                }
+            }
+            if (have) {                             // CTA-uniform per stream: every thread of the warpgroup posts
+                EpiMsg* msg = &sc->epi[msg_n & 1u];
+                msg->inv[row] = inv;
+                if (row == 0) {
+                    msg->kind = kEpiTile;
+                    msg->bh = slot->bh;
+                    msg->qa = slot->qa;
+                    msg->qb = slot->qb;
+                    msg->part_slot = part_slot;
+                }
+                mbar_arrive(&sc->epi_full[msg_n & 1u]);      // (release: the message is visible to whoever sees the phase complete)
+                ++msg_n;
+            }
+        }
+        tc_fence_before();
+        mbar_arrive(&sc->sched_empty[ss]);
+        ++sched_n;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------ epilogue (one warpgroup, both streams)
+// Each warp serves its 32 rows of whichever stream has a finished tile: accumulator out of tensor memory,
+// scaled by 1/l, to the output rows (or raw, to the scratch of a split tile's part).
+__device__ __forceinline__ void epilogue_role(const KernelParams& p, SmemCtl* ctl, unsigned char* smem, unsigned tmem, int warp, int lane) {
+    int* abort_flag = &ctl->abort_flag;
+    const int quad = warp & 3;
+    const int row = quad * 32 + lane;
+    const int r64 = row & (kBlock - 1);
+    const bool lower = row >= kBlock;
+    // per stream, packed so that the loop below is one copy of the code: bits 0..15 messages taken, 16..30 tiles
+    // taken (only parities are used), bit 31 the stream is finished
+    unsigned state[kStreams] = {0u, 0u};
+    IdleClock idle;
+    while (!((state[0] & state[1]) >> 31)) {
+        bool progress = false;
+#pragma unroll 1
+        for (int s = 0; s < kStreams; ++s) {
+            const unsigned st = state[s];
+            if (st >> 31) continue;
+            StreamCtl* sc = &ctl->st[s];
+            const unsigned msg_n = st & 0xffffu, tile_n = (st >> 16) & 0x7fffu;
+            const unsigned e = msg_n & 1u, eph = (msg_n >> 1) & 1u;
+            if (!__all_sync(0xffffffffu, mbar_test(&sc->epi_full[e], eph))) continue;
+            progress = true;
+            const EpiMsg* msg = &sc->epi[e];
+            if (msg->kind == kEpiDone) { state[s] = st | 0x80000000u; continue; }
+            state[s] = ((msg_n + 1u) & 0xffffu) | (((tile_n + 1u) & 0x7fffu) << 16);
+            const int bh = msg->bh, my_q = lower ? msg->qb : msg->qa, part_slot = msg->part_slot;
+            const float inv = msg->inv[row];
+            if (!mbar_wait(&sc->o_done, tile_n & 1u, abort_flag, p.status, 40)) return;
+            tc_fence_after();
+            const unsigned lane_addr = tmem + s * kStreamCols + ((unsigned)(quad * 32) << 16);
+            // the row's destination: the output tensor, or (raw fp32) the scratch of a split tile's part
+            const bool partial = part_slot >= 0;
+            unsigned char* dst = partial ? reinterpret_cast<unsigned char*>(p.partials + (size_t)part_slot * kPartialFloats + row * 64)
+                                         : reinterpret_cast<unsigned char*>(p.out + (((size_t)bh * p.nb + (my_q >= 0 ? my_q : 0)) * kBlock + r64) * kBlock);
+            const bool write = partial || my_q >= 0;        // warp-uniform
+#pragma unroll 1
+            for (int c = 0; c < 2; ++c) {
+                float o[32];
+                tmem_ld32(lane_addr + kColO + c * 32, o);
+                tmem_wait_ld();
+                if (c == 1) { tc_fence_before(); mbar_arrive(&sc->o_free); }       // the accumulator has been taken
+                if (!write) continue;
+                if (partial) {
+                    float4* d4 = reinterpret_cast<float4*>(dst) + 8 * c;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) d4[j] = make_float4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+                } else {
+                    uint4* d4 = reinterpret_cast<uint4*>(dst) + 4 * c;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        uint4 v;
+                        v.x = pack_bf16(o[8 * j + 0] * inv, o[8 * j + 1] * inv);
+                        v.y = pack_bf16(o[8 * j + 2] * inv, o[8 * j + 3] * inv);
+                        v.z = pack_bf16(o[8 * j + 4] * inv, o[8 * j + 5] * inv);
+                        v.w = pack_bf16(o[8 * j + 6] * inv, o[8 * j + 7] * inv);
+                        d4[j] = v;
+                    }
+                }
+            }
+        }
+        if (progress) idle.reset();
+        else {
+            // suspended on stream 0's next message for a short while; stream 1's is looked at again afterwards
+            const unsigned st0 = state[0];
+            if (!(st0 >> 31)) mbar_try_for(&ctl->st[0].epi_full[st0 & 1u], (st0 >> 1) & 1u, 300);
+            else __nanosleep(300);
+            if (!__all_sync(0xffffffffu, idle.tick(abort_flag, p.status, 41, 0))) return;
+        }
+    }
+}
+
 // ------------------------------------------------------------------------------------------------ the kernel
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, 1)
 attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                       const __grid_constant__ CUtensorMap tm_v, const KernelParams p) {
     extern __shared__ unsigned char smem_raw[];
@@ -325,18 +1006,23 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < kRingGroups; ++i) { mbar_init(&ctl->full[i], 1); mbar_init(&ctl->empty[i], 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(&ctl->q_full[i], 1); mbar_init(&ctl->q_empty[i], 1); }
-        mbar_init(&ctl->s_full, 1);
-        mbar_init(&ctl->s_free, kSoftmaxWarps * 32);    // every softmax thread arrives itself: cheaper than
-        mbar_init(&ctl->p_full, kSoftmaxWarps * 32);    // converging the warp and electing a lane
-        mbar_init(&ctl->pv_done, 1);
-        for (int i = 0; i < kSchedSlots; ++i) { mbar_init(&ctl->sched_full[i], 1); mbar_init(&ctl->sched_empty[i], 2 + kSoftmaxWarps * 32); }
+        for (int s = 0; s < kStreams; ++s) {
+            StreamCtl* sc = &ctl->st[s];
+            for (int i = 0; i < kRingGroups; ++i) { mbar_init(&sc->full[i], 1); mbar_init(&sc->empty[i], 1); }
+            for (int i = 0; i < 2; ++i) { mbar_init(&sc->q_full[i], 1); mbar_init(&sc->q_empty[i], 1); mbar_init(&sc->epi_full[i], kSoftmaxThreads); }
+            mbar_init(&sc->s_full, 1);
+            mbar_init(&sc->s_free, kSoftmaxThreads);    // every softmax thread arrives itself: cheaper than
+            mbar_init(&sc->p_full, kSoftmaxThreads);    // converging the warp and electing a lane
+            mbar_init(&sc->pv_done, 1);
+            mbar_init(&sc->o_done, 1);
+            mbar_init(&sc->o_free, kSoftmaxThreads);    // the 128 epilogue threads
+            for (int i = 0; i < kSchedSlots; ++i) { mbar_init(&sc->sched_full[i], 1); mbar_init(&sc->sched_empty[i], 2 + kSoftmaxThreads); }
+        }
         ctl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 1) {
+    if (warp == kWarpProducer) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -344,435 +1030,20 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     __syncthreads();
     tc_fence_after();
     const unsigned tmem = *(volatile unsigned*)&ctl->tmem_base;
+    const StreamRef s0{&ctl->st[0], smem, tmem};
+    const StreamRef s1{&ctl->st[1], smem + kStreamSmemBytes, tmem + kStreamCols};
 
-    if (warp < 4) {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsLight));
-        if (warp == 2) {
-            // ================================================================= scheduler: fetch work, post live key blocks
-            unsigned sched_n = 0;
-            bool ok = true;
-            const unsigned lt_mask = (1u << lane) - 1u;
-            while (ok) {
-                int w = 0;
-                if (lane == 0) w = atomicAdd(&p.counter[0], 1);
-                w = __shfl_sync(0xffffffffu, w, 0);
-                if (w >= p.total_work) w = -1;
-                // decode the work index: global-row tiles of every (batch, head) first, then the sparse tiles
-                int bh = 0, it = 0;
-                Item item{};
-                if (w >= 0) {
-                    const int heavy_total = p.BH * p.heavy_per_head;
-                    if (w < heavy_total) {
-                        bh = w / p.heavy_per_head;
-                        it = w - bh * p.heavy_per_head;
-                    } else {
-                        const int sparse = p.items_per_head - p.heavy_per_head;
-                        const int w2 = w - heavy_total;
-                        bh = w2 / sparse;
-                        it = p.heavy_per_head + (w2 - bh * sparse);
-                    }
-                    item = p.items[(size_t)(bh % p.H) * p.items_per_head + it];
-                }
-                const int batch = bh / p.H;
-                const unsigned long long qbits_a = w >= 0 ? key_bits(p, batch, item.qa) : 0ull;
-                const unsigned long long qbits_b = w >= 0 ? key_bits(p, batch, item.qb) : 0ull;
-                const bool tile_live = (qbits_a | qbits_b) != 0ull;      // a tile whose query rows are all padding is skipped
-                const int n_raw = (w >= 0 && tile_live) ? item.step_count : 0;
-                int i0 = 0;
-                bool first = true;
-                do {
-                    const unsigned ss = sched_n % kSchedSlots, sp = (sched_n / kSchedSlots) & 1u;
-                    ok = mbar_wait(&ctl->sched_empty[ss], sp ^ 1u, ctl, p.status, 11);
-                    if (!ok) break;
-                    WorkSlot* slot = &ctl->slot[ss];
-                    int count = 0;
-                    while (i0 < n_raw && count <= kSegChunks - 32) {
-                        const int i = i0 + lane;
-                        ChunkEntry e{-1, 0, 0ull};
-                        bool alive = false;
-                        if (i < n_raw) {
-                            const Step s = p.steps[item.step_begin + i];
-                            // halves whose query rows are all padding do not attend anything
-                            const bool ua = s.who != kLowerHalf && qbits_a != 0ull;
-                            const bool ub = s.who != kUpperHalf && qbits_b != 0ull;
-                            e.c = s.c;
-                            e.kb = key_bits(p, batch, s.c);
-                            e.who = ((ua && ub) ? kBothHalves : (ua ? kUpperHalf : kLowerHalf)) | (e.kb != ~0ull ? kHasPadding : 0);
-                            alive = e.kb != 0ull && (ua || ub);
-                        }
-                        const unsigned bal = __ballot_sync(0xffffffffu, alive);
-                        if (alive) slot->chunks[count + __popc(bal & lt_mask)] = e;
-                        count += __popc(bal);
-                        i0 += 32;
-                    }
-                    if (lane == 0) {
-                        slot->w = w;
-                        slot->bh = bh;
-                        slot->batch = batch;
-                        slot->qa = item.qa;
-                        slot->qb = item.qb;
-                        slot->n_chunks = count;
-                        slot->flags = (first ? kSegFirst : 0) | (i0 >= n_raw ? kSegLast : 0) | (tile_live ? kSegLive : 0);
-                        slot->qbits_a = qbits_a;
-                        slot->qbits_b = qbits_b;
-                        slot->part_slot = (w >= 0 && item.nparts > 1) ? ((bh * p.split_tiles_per_head + item.tile) * p.max_parts + item.part) : -1;
-                    }
-                    __threadfence_block();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&ctl->sched_full[ss]);
-                    ++sched_n;
-                    first = false;
-                } while (i0 < n_raw);
-                if (w < 0) break;
-            }
-        } else if (warp == 0 && lane == 0) {
-            // ================================================================= TMA producer
-            // Ring order = the order in which the MMA thread consumes groups: K of step i, then V of step i-1.
-            unsigned ring_n = 0, q_n = 0, sched_n = 0;
-            bool ok = true;
-            // the (up to two) blocks c[0..cnt) of K or V into the next group of adjacent ring slots
-            auto load_group = [&](const CUtensorMap* tm, int bh, const int* c, int cnt) -> bool {
-                const unsigned g = ring_n % kRingGroups, ph = (ring_n / kRingGroups) & 1u;
-                if (!mbar_wait(&ctl->empty[g], ph ^ 1u, ctl, p.status, 10)) return false;
-                mbar_expect_tx(&ctl->full[g], cnt * kTileBytes);
-#pragma unroll
-                for (int j = 0; j < kStepChunks; ++j)
-                    if (j < cnt) tma_load_tile(smem + kSmemRing + g * kGroupBytes + j * kTileBytes, tm, (bh * p.nb + c[j]) * kBlock, &ctl->full[g]);
-                ++ring_n;
-                return true;
-            };
-            int pend_n = 0, pend_bh = 0, pend_c[kStepChunks] = {0, 0};
-            while (ok) {
-                const unsigned ss = sched_n % kSchedSlots, sp = (sched_n / kSchedSlots) & 1u;
-                if (!mbar_wait(&ctl->sched_full[ss], sp, ctl, p.status, 13)) break;
-                const WorkSlot* slot = &ctl->slot[ss];
-                const int w = slot->w, flags = slot->flags, bh = slot->bh, n = slot->n_chunks;
-                if (w >= 0 && (flags & kSegLive)) {
-                    if (flags & kSegFirst) {
-                        const int qa = slot->qa, qb = slot->qb;
-                        const unsigned qs = q_n & 1u;
-                        ok = mbar_wait(&ctl->q_empty[qs], ((q_n >> 1) & 1u) ^ 1u, ctl, p.status, 12);
-                        if (!ok) break;
-                        mbar_expect_tx(&ctl->q_full[qs], qb >= 0 ? 2 * kTileBytes : kTileBytes);
-                        tma_load_tile(smem + kSmemQ + qs * 2 * kTileBytes, &tm_q, (bh * p.nb + qa) * kBlock, &ctl->q_full[qs]);
-                        if (qb >= 0) tma_load_tile(smem + kSmemQ + qs * 2 * kTileBytes + kTileBytes, &tm_q, (bh * p.nb + qb) * kBlock, &ctl->q_full[qs]);
-                        ++q_n;
-                    }
-                    for (int i = 0; i < n && ok; i += kStepChunks) {
-                        int c[kStepChunks];
-                        const int cnt = min(kStepChunks, n - i);
-#pragma unroll
-                        for (int j = 0; j < kStepChunks; ++j) c[j] = j < cnt ? slot->chunks[i + j].c : 0;
-                        ok = load_group(&tm_k, bh, c, cnt);
-                        if (ok && pend_n > 0) ok = load_group(&tm_v, pend_bh, pend_c, pend_n);
-#pragma unroll
-                        for (int j = 0; j < kStepChunks; ++j) pend_c[j] = c[j];
-                        pend_n = cnt;
-                        pend_bh = bh;
-                    }
-                }
-                mbar_arrive(&ctl->sched_empty[ss]);
-                ++sched_n;
-                if (w < 0) {
-                    if (ok && pend_n > 0) load_group(&tm_v, pend_bh, pend_c, pend_n);
-                    break;
-                }
-            }
-        } else if (warp == 1 && lane == 0) {
-            // ================================================================= MMA issuer
-            unsigned ring_n = 0, q_n = 0, sched_n = 0, grp_n = 0, pv_n = 0;   // grp_n: steps whose Q K^T was issued
-            bool ok = true;
-            auto qk = [&](int cnt, unsigned qs) -> bool {   // S[:, 0 .. 64 cnt) = Q K^T with the K blocks of the next ring group
-                const unsigned g = ring_n % kRingGroups, ph = (ring_n / kRingGroups) & 1u;
-                if (!mbar_wait(&ctl->full[g], ph, ctl, p.status, 20)) return false;
-                tc_fence_after();
-                // the blocks of a group are adjacent: their 64 cnt rows form one K-major operand
-                const unsigned long long q_desc = smem_desc_sw128(smem_u32(smem + kSmemQ + qs * 2 * kTileBytes));
-                const unsigned long long k_desc = smem_desc_sw128(smem_u32(smem + kSmemRing + g * kGroupBytes));
-                const unsigned idesc = kIdescQK64 + ((unsigned)(cnt - 1) << 20);           // N = 64 cnt
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk)          // 16 head dims (32 bytes inside the swizzled row) per MMA
-                    mma_ss(tmem + kColS, q_desc + (unsigned long long)(kk * 2), k_desc + (unsigned long long)(kk * 2), idesc, kk > 0);
-                tc_commit(&ctl->empty[g]);
-                ++ring_n;
-                return true;
-            };
-            bool pend_fresh = false;                    // the pending P V is the first of its tile: it overwrites O
-            bool tile_fresh = false, q_unseen = false;
-            int pend_n = 0;
-            auto pending_pv = [&]() -> bool {           // O (+)= sum_j P_j V_j with the V blocks of the next ring group
-                if (pend_n == 0) return true;
-                if (!mbar_wait(&ctl->p_full, pv_n & 1u, ctl, p.status, 22)) return false;
-                const unsigned g = ring_n % kRingGroups, ph = (ring_n / kRingGroups) & 1u;
-                if (!mbar_wait(&ctl->full[g], ph, ctl, p.status, 21)) return false;
-                tc_fence_after();
-                const unsigned long long v_desc = smem_desc_sw128(smem_u32(smem + kSmemRing + g * kGroupBytes));
-#pragma unroll
-                for (int j = 0; j < kStepChunks; ++j) {
-                    if (j < pend_n) {
-#pragma unroll
-                        for (int kk = 0; kk < 4; ++kk)  // 16 keys per MMA: 8 packed columns of P_j, two 8-row groups of V_j
-                            mma_ts(tmem + kColO, tmem + kColP + 32 * j + kk * 8, v_desc + (unsigned long long)((j * kTileBytes + kk * 2048) >> 4), kIdescPV,
-                                   (j > 0 || kk > 0 || !pend_fresh) ? 1u : 0u);
-                    }
-                }
-                tc_commit(&ctl->empty[g]);
-                tc_commit(&ctl->pv_done);
-                ++ring_n;
-                ++pv_n;
-                pend_n = 0;
-                pend_fresh = false;
-                return true;
-            };
-            while (ok) {
-                const unsigned ss = sched_n % kSchedSlots, sp = (sched_n / kSchedSlots) & 1u;
-                if (!mbar_wait(&ctl->sched_full[ss], sp, ctl, p.status, 23)) break;
-                const WorkSlot* slot = &ctl->slot[ss];
-                const int w = slot->w, flags = slot->flags, n = slot->n_chunks;
-                if (w >= 0 && (flags & kSegLive)) {
-                    if (flags & kSegFirst) {
-                        ++q_n;                          // this tile's Q sits in buffer (q_n - 1) & 1
-                        q_unseen = true;
-                        tile_fresh = true;
-                    }
-                    const unsigned qs = (q_n - 1) & 1u, qph = ((q_n - 1) >> 1) & 1u;
-                    for (int i = 0; i < n && ok; i += kStepChunks) {
-                        // the softmax threads must have pulled the previous scores out of tensor memory
-                        if (grp_n > 0) {
-                            ok = mbar_wait(&ctl->s_free, (grp_n - 1) & 1u, ctl, p.status, 25);
-                            if (!ok) break;
-                        }
-                        if (q_unseen) {
-                            ok = mbar_wait(&ctl->q_full[qs], qph, ctl, p.status, 24);
-                            if (!ok) break;
-                            q_unseen = false;
-                        }
-                        tc_fence_after();
-                        const int cnt = min(kStepChunks, n - i);
-                        ok = qk(cnt, qs);
-                        if (!ok) break;
-                        tc_commit(&ctl->s_full);
-                        ++grp_n;
-                        // the previous step's P V goes behind this step's Q K^T
-                        ok = pending_pv();
-                        pend_n = cnt;
-                        pend_fresh = tile_fresh;
-                        tile_fresh = false;
-                    }
-                    if (!ok) break;
-                    if (flags & kSegLast) {
-                        if (q_unseen) {                 // a tile without a live key block: its Q still has to land
-                            ok = mbar_wait(&ctl->q_full[qs], qph, ctl, p.status, 26);
-                            if (!ok) break;
-                            q_unseen = false;
-                        }
-                        tc_commit(&ctl->q_empty[qs]);   // every Q K^T of the tile has been issued
-                    }
-                }
-                mbar_arrive(&ctl->sched_empty[ss]);
-                ++sched_n;
-                if (w < 0) {
-                    pending_pv();
-                    break;
-                }
-            }
-        }
-    } else {
+    if (warp < kWarpEpilogue) {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
-        // ===================================================================== softmax + epilogue (128 threads, one per row)
-        const int quad = warp & 3;                      // tensor-memory lanes this warp may touch: 32*quad .. +31
-        const int row = quad * 32 + lane;               // row of the 128-row tile
-        const bool lower = row >= kBlock;
-        const int my_who = lower ? kLowerHalf : kUpperHalf;
-        const unsigned lane_addr = tmem + ((unsigned)(quad * 32) << 16);
-        const float sl2 = p.scale_log2;
-        unsigned sched_n = 0, grp_n = 0;
-        bool ok = true;
-        float m_ref = -INFINITY, l_sum = 0.f;
-        bool o_dirty = false;                           // has any P V been issued for this tile yet
-        // output of the previous tile, written once its last P V is known to be complete
-        bool pend_out = false, pend_partial = false;
-        float pend_inv = 0.f;
-        uint4* pend_dst = nullptr;
-        auto write_out = [&]() {                        // the 64 accumulator columns of this thread's row
-#pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                float o[32];
-                tmem_ld32(lane_addr + kColO + c * 32, o);
-                tmem_wait_ld();
-                if (pend_partial) {                     // one part of a split tile: the raw fp32 accumulator
-                    float4* d4 = reinterpret_cast<float4*>(pend_dst) + 8 * c;
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) d4[j] = make_float4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
-                } else {                                // pend_inv is 0 for rows that must come out as zeros
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        uint4 v4;
-                        v4.x = pack_bf16(o[8 * j + 0] * pend_inv, o[8 * j + 1] * pend_inv);
-                        v4.y = pack_bf16(o[8 * j + 2] * pend_inv, o[8 * j + 3] * pend_inv);
-                        v4.z = pack_bf16(o[8 * j + 4] * pend_inv, o[8 * j + 5] * pend_inv);
-                        v4.w = pack_bf16(o[8 * j + 6] * pend_inv, o[8 * j + 7] * pend_inv);
-                        pend_dst[4 * c + j] = v4;
-                    }
-                }
-            }
-            pend_out = false;
-        };
-        // -inf over the scores of padded keys of one key block, in tensor memory (s: 64 scratch registers)
-        auto mask_scores = [&](float* s, unsigned taddr, unsigned long long kb) {
-            tmem_ld64(taddr, s);
-            tmem_wait_ld();
-#pragma unroll
-            for (int t = 0; t < 64; ++t) s[t] = ((kb >> t) & 1ull) ? s[t] : -INFINITY;
-            tmem_st32(taddr, reinterpret_cast<unsigned*>(s));
-            tmem_st32(taddr + 32, reinterpret_cast<unsigned*>(s + 32));
-            tmem_wait_st();
-        };
-        // exponentials of the 64 scores of one key block, packed in place: afterwards s[0..31] hold the bit
-        // patterns of the 32 words of bf16 probability pairs
-        auto exp_pack = [&](float* s, float neg_m, float& sum0, float& sum1) {
-#pragma unroll
-            for (int t = 0; t < 64; t += 2) {
-                float t0, t1;
-                ffma2(t0, t1, s[t], s[t + 1], sl2, neg_m);
-                const float p0 = ex2(t0), p1 = ex2(t1);
-                fadd2(sum0, sum1, p0, p1);
-                s[t >> 1] = __uint_as_float(pack_bf16(p0, p1));
-            }
-        };
-        while (ok) {
-            const unsigned ss = sched_n % kSchedSlots, sp = (sched_n / kSchedSlots) & 1u;
-            if (!mbar_wait(&ctl->sched_full[ss], sp, ctl, p.status, 30)) break;
-            const WorkSlot* slot = &ctl->slot[ss];
-            const int w = slot->w, flags = slot->flags, n = slot->n_chunks;
-            if (w < 0) {
-                if (pend_out) {                         // warp-uniform; the last P V of all
-                    ok = mbar_wait(&ctl->pv_done, (grp_n - 1) & 1u, ctl, p.status, 35);
-                    if (!ok) break;
-                    tc_fence_after();
-                    write_out();
-                }
-                break;
-            }
-            const bool live = flags & kSegLive;
-            if (flags & kSegFirst) {
-                m_ref = -INFINITY;
-                l_sum = 0.f;
-                o_dirty = false;
-            }
-            for (int i = 0; i < n && ok; i += kStepChunks) {
-                const ChunkEntry* e = &slot->chunks[i];
-                const int cnt = min(kStepChunks, n - i);
-                // which of the step's key blocks my half of the tile attends (warp-uniform)
-                const int who0 = e[0].who, who1 = cnt > 1 ? e[1].who : kNoChunk;
-                const bool mine0 = (who0 & kWhoMask) == kBothHalves || (who0 & kWhoMask) == my_who;
-                const bool mine1 = (who1 & kWhoMask) == kBothHalves || (who1 & kWhoMask) == my_who;
-                ok = mbar_wait(&ctl->s_full, grp_n & 1u, ctl, p.status, 31);
-                if (!ok) break;
-                tc_fence_after();
-                float s[128];
-                // A key block with padded keys (rare: the one holding a sequence's end) gets -inf written over their
-                // scores in tensor memory first, so that the common path below carries no masking code at all.
-                if (__builtin_expect(((who0 | who1) & kHasPadding) != 0, 0)) {
-                    if (mine0 && (who0 & kHasPadding)) mask_scores(s, lane_addr + kColS, e[0].kb);
-                    if (mine1 && (who1 & kHasPadding)) mask_scores(s, lane_addr + kColS + 64, e[1].kb);
-                }
-                if (mine0) tmem_ld64(lane_addr + kColS, s);
-                if (mine1) tmem_ld64(lane_addr + kColS + 64, s + 64);
-                tmem_wait_ld();
-                // the score columns are free again: the next step's Q K^T may overwrite them
-                tc_fence_before();
-                mbar_arrive(&ctl->s_free);
-                float alpha = 1.f;
-                bool rescale = false;
-                if (mine0 || mine1) {
-                    float m_loc = -INFINITY;
-                    if (mine0) m_loc = row_max64(s);
-                    if (mine1) m_loc = fmaxf(m_loc, row_max64(s + 64));
-                    const float m_cand = m_loc * sl2;
-                    const bool need = m_cand > m_ref + kRescaleThreshold;        // true on the first step (m_ref = -inf)
-                    rescale = __any_sync(0xffffffffu, need);
-                    if (need) {
-                        alpha = ex2(m_ref - m_cand);
-                        m_ref = m_cand;
-                    }
-                }
-                // probabilities into registers first: the previous step's P V has this long to finish
-                float sum0 = 0.f, sum1 = 0.f;
-                const float neg_m = -m_ref;
-                if (mine0) exp_pack(s, neg_m, sum0, sum1);
-                if (mine1) exp_pack(s + 64, neg_m, sum0, sum1);
-                // the previous step's P V must be complete before its probabilities are overwritten or O is touched
-                if (grp_n > 0) {
-                    ok = mbar_wait(&ctl->pv_done, (grp_n - 1) & 1u, ctl, p.status, 32);
-                    if (!ok) break;
-                    tc_fence_after();
-                }
-                if (__builtin_expect(pend_out, 0)) write_out();      // warp-uniform: the previous tile's accumulator is complete
-                if (__builtin_expect(rescale && o_dirty, 0)) {
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        float o[16];
-                        tmem_ld16(lane_addr + kColO + c * 16, o);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int t = 0; t < 16; t += 2) fmul2(o[t], o[t + 1], alpha);
-                        tmem_st16(lane_addr + kColO + c * 16, reinterpret_cast<unsigned*>(o));
-                    }
-                }
-                if (mine0) tmem_st32(lane_addr + kColP, reinterpret_cast<unsigned*>(s));
-                else tmem_st32_zero(lane_addr + kColP);
-                if (cnt > 1) {
-                    if (mine1) tmem_st32(lane_addr + kColP + 32, reinterpret_cast<unsigned*>(s + 64));
-                    else tmem_st32_zero(lane_addr + kColP + 32);
-                }
-                l_sum = l_sum * alpha + (sum0 + sum1);
-                tmem_wait_st();
-                tc_fence_before();
-                mbar_arrive(&ctl->p_full);
-                ++grp_n;
-                o_dirty = true;
-            }
-            if (!ok) break;
-            if (flags & kSegLast) {
-                // -------------------------------------------------------- end of the tile: lse, output pointer
-                const int my_q = lower ? slot->qb : slot->qa;
-                const unsigned long long qbits = lower ? slot->qbits_b : slot->qbits_a;
-                const bool have = live && o_dirty;
-                const int part_slot = slot->part_slot;
-                if (part_slot >= 0) {
-                    // one part of a split tile: (max, sum) now, the accumulator once its last P V is complete
-                    float* part = p.partials + (size_t)part_slot * kPartialFloats;
-                    part[128 * 64 + row] = have ? m_ref : -INFINITY;
-                    part[128 * 64 + 128 + row] = have ? l_sum : 0.f;
-                    if (have) {
-                        pend_out = true;
-                        pend_partial = true;
-                        pend_dst = reinterpret_cast<uint4*>(part + row * 64);
-                    }
-                } else if (my_q >= 0) {                 // warp-uniform
-                    const int r64 = row & (kBlock - 1);
-                    const bool good = have && ((qbits >> r64) & 1ull) && l_sum > 0.f;
-                    const size_t tok = ((size_t)slot->bh * p.nb + my_q) * kBlock + r64;
-                    uint4* dst = reinterpret_cast<uint4*>(p.out + tok * kBlock);
-                    if (p.lse) p.lse[tok] = good ? (m_ref + __log2f(l_sum)) * 0.6931471805599453f : -INFINITY;
-                    if (have) {
-                        // the accumulator is read once the tile's last P V is known to be complete
-                        pend_out = true;
-                        pend_partial = false;
-                        pend_inv = good ? __frcp_rn(l_sum) : 0.f;
-                        pend_dst = dst;
-                    } else {
-                        const uint4 z = make_uint4(0u, 0u, 0u, 0u);
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) dst[j] = z;
-                    }
-                }
-            }
-            tc_fence_before();
-            mbar_arrive(&ctl->sched_empty[ss]);
-            ++sched_n;
-        }
+        softmax_role(p, ctl, warp < 4 ? s0 : s1, warp, lane);
+    } else if (warp < kWarpProducer) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsEpilogue));
+        epilogue_role(p, ctl, smem, tmem, warp, lane);
+    } else {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsLight));
+        if (warp == kWarpScheduler) scheduler_role(p, ctl, lane);
+        else if (warp == kWarpProducer) { if (lane < kStreams) producer_role(p, ctl, lane == 0 ? s0 : s1, &tm_q, &tm_k, &tm_v); }
+        else if (lane == 0) mma_role(p, ctl, warp == kWarpMma ? s0 : s1);
     }
 
     // ------------------------------------------------------------------------------------------------ teardown
@@ -784,7 +1055,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         __syncthreads();
     }
     tc_fence_after();
-    if (warp == 1) {
+    if (warp == kWarpProducer) {
         __syncwarp();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
@@ -840,14 +1111,13 @@ merge_split_tiles_kernel(const float* __restrict__ partials, const int* __restri
 // helper and the same limit as the attention kernel; the wait gives up, records BIGBIRD_ETIMEOUT and the kernel
 // returns normally.
 __global__ void wait_expiry_selftest_kernel(int* status) {
-    extern __shared__ unsigned char smem_raw[];
-    unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    SmemCtl* ctl = reinterpret_cast<SmemCtl*>(smem + kSmemCtl);
+    __shared__ unsigned long long bar;
+    __shared__ int abort_flag;
     if (threadIdx.x == 0) {
-        mbar_init(&ctl->s_full, 1);
-        ctl->abort_flag = 0;
+        mbar_init(&bar, 1);
+        abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        mbar_wait(&ctl->s_full, 0u, ctl, status, 99);
+        mbar_wait(&bar, 0u, &abort_flag, status, 99);
     }
 }
 
@@ -896,11 +1166,46 @@ bool make_map(CUtensorMap* tm, const void* base, uint64_t rows) {
 }  // namespace
 
 cudaError_t launch_wait_expiry_selftest(DeviceScratch& sc, cudaStream_t stream) {
-    cudaError_t e = cudaFuncSetAttribute(wait_expiry_selftest_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-    if (e != cudaSuccess) return e;
-    wait_expiry_selftest_kernel<<<1, 32, kSmemBytes, stream>>>(sc.status);
+    wait_expiry_selftest_kernel<<<1, 32, 0, stream>>>(sc.status);
     return cudaGetLastError();
 }
+
+namespace {
+
+// Per device, once, with that device current: the kernel's shared-memory attribute (a per-device property of the
+// function) and the device's SM count.
+struct KernelDevice {
+    bool ready = false;
+    int sm_count = 0;
+};
+constexpr int kMaxKernelDevices = 64;
+std::mutex g_kernel_mu, g_launch_mu;
+KernelDevice g_kernel_dev[kMaxKernelDevices];
+
+cudaError_t kernel_setup(int device, int* sm_count) {
+    if (device < 0 || device >= kMaxKernelDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_kernel_mu);
+    KernelDevice& d = g_kernel_dev[device];
+    if (!d.ready) {
+        cudaError_t e = cudaFuncSetAttribute(attn_fwd_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e != cudaSuccess) return e;
+        e = cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, device);
+        if (e != cudaSuccess) return e;
+        d.ready = true;
+    }
+    *sm_count = d.sm_count;
+    return cudaSuccess;
+}
+
+// One CTA per SM, each running kStreams tile streams.
+int grid_size(int sm_count, int total_work) {
+    int grid = sm_count;
+    const int needed = (total_work + kStreams - 1) / kStreams;
+    if (grid > needed) grid = needed;
+    return grid < 1 ? 1 : grid;
+}
+
+}  // namespace
 
 int launch_attn_fwd_sm100(const FwdArgs& a, const bigbird_layout& L, const DeviceLayout& dl, DeviceScratch& sc,
                           int* launches, cudaError_t* cuda_err) {
@@ -909,16 +1214,13 @@ int launch_attn_fwd_sm100(const FwdArgs& a, const bigbird_layout& L, const Devic
     const int64_t rows = (int64_t)a.B * a.H * a.N;
     if (rows >= (1ll << 31) || (int64_t)a.B * a.H * L.items_per_head >= (1ll << 31)) return BIGBIRD_EUNSUPPORTED;
 
-    static std::once_flag attr_once;
-    static cudaError_t attr_err = cudaSuccess;
-    static int sm_count = 0;
-    std::call_once(attr_once, [] {
-        attr_err = cudaFuncSetAttribute(attn_fwd_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-        int dev = 0;
-        if (attr_err == cudaSuccess) attr_err = cudaGetDevice(&dev);
-        if (attr_err == cudaSuccess) attr_err = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-    });
-    if (attr_err != cudaSuccess) { *cuda_err = attr_err; return BIGBIRD_ECUDA; }
+    // One host thread at a time past this point: the per-device scratch bookkeeping below (counter slots, grown
+    // buffers) is plain data.
+    std::lock_guard<std::mutex> launch_lock(g_launch_mu);
+    int device = 0, sm_count = 0;
+    cudaError_t de = cudaGetDevice(&device);
+    if (de == cudaSuccess) de = kernel_setup(device, &sm_count);
+    if (de != cudaSuccess) { *cuda_err = de; return BIGBIRD_ECUDA; }
 
     CUtensorMap tm_q, tm_k, tm_v;
     if (!make_map(&tm_q, a.q, (uint64_t)rows) || !make_map(&tm_k, a.k, (uint64_t)rows) || !make_map(&tm_v, a.v, (uint64_t)rows)) {
@@ -977,9 +1279,7 @@ int launch_attn_fwd_sm100(const FwdArgs& a, const bigbird_layout& L, const Devic
     p.total_work = p.BH * L.items_per_head;
     p.scale_log2 = a.scale * 1.4426950408889634f;
 
-    int grid = 2 * sm_count;
-    if (grid > p.total_work) grid = p.total_work;
-    if (grid < 1) grid = 1;
+    const int grid = grid_size(sm_count, p.total_work);
     attn_fwd_sm100_kernel<<<grid, kThreads, kSmemBytes, a.stream>>>(tm_q, tm_k, tm_v, p);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { *cuda_err = e; return BIGBIRD_ECUDA; }
@@ -1000,7 +1300,7 @@ int launch_attn_fwd_sm100(const FwdArgs& a, const bigbird_layout& L, const Devic
 // bigbird_attn_fwd_static: the tensor-core forward for callers that must not allocate device memory (see
 // include/bigbird.h).  Everything bigbird_attn_fwd keeps in cudaMalloc'ed library scratch lives here in one
 // fixed array that is part of the loaded module: status and work-counter words, the packed key-padding bits,
-// and the device copy of the layout's tile schedule, which is re-sent on every call.
+// and the device copy of the layout's tile schedule, which is sent again whenever another layout is used.
 namespace bigbird {
 namespace {
 
@@ -1017,6 +1317,7 @@ static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
 struct StaticDevice {
     unsigned char* base = nullptr;              // device address of g_static_scratch on this device
     int sm_count = 0;
+    uint64_t schedule_uid = 0;                  // layout whose schedule the array holds (0: none)
 };
 std::mutex g_static_mu;
 StaticDevice g_static_dev[64];
@@ -1030,10 +1331,8 @@ cudaError_t static_setup(int device, StaticDevice* out) {
         void* ptr = nullptr;
         cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(attn_fwd_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-        if (e != cudaSuccess) return e;
         int sms = 0;
-        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+        e = kernel_setup(device, &sms);
         if (e != cudaSuccess) return e;
         d.sm_count = sms;
         d.base = (unsigned char*)ptr;
@@ -1041,6 +1340,12 @@ cudaError_t static_setup(int device, StaticDevice* out) {
     *out = d;
     return cudaSuccess;
 }
+
+void static_remember_schedule(int device, uint64_t uid) {
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    g_static_dev[device].schedule_uid = uid;
+}
+void static_forget_schedule(int device) { static_remember_schedule(device, 0); }
 
 }  // namespace
 }  // namespace bigbird
@@ -1082,13 +1387,14 @@ extern "C" int bigbird_attn_fwd_static(const void* q, const void* k, const void*
     // this call's layout replaces the previous one (step offsets made absolute, as the kernel expects).
     e = cudaMemsetAsync(words4, 0, 16, stream);
     if (e != cudaSuccess) return BIGBIRD_ECUDA;
-    static thread_local std::vector<Item> items_abs;            // host memory only
-    items_abs = L->items;
-    for (int h = 0; h < L->H; ++h)
-        for (int i = 0; i < L->items_per_head; ++i) items_abs[(size_t)h * L->items_per_head + i].step_begin += L->step_base[h];
-    e = cudaMemcpyAsync(items_dev, items_abs.data(), n_items * sizeof(Item), cudaMemcpyHostToDevice, stream);
-    if (e == cudaSuccess && n_steps) e = cudaMemcpyAsync(steps_dev, L->steps.data(), n_steps * sizeof(Step), cudaMemcpyHostToDevice, stream);
-    if (e != cudaSuccess) return BIGBIRD_ECUDA;
+    // The schedule is sent only when the array does not hold this layout's already (copies from the handle's own
+    // host arrays, which live as long as the handle).
+    if (sd.schedule_uid != L->uid) {
+        e = cudaMemcpyAsync(items_dev, L->items_abs.data(), n_items * sizeof(Item), cudaMemcpyHostToDevice, stream);
+        if (e == cudaSuccess && n_steps) e = cudaMemcpyAsync(steps_dev, L->steps.data(), n_steps * sizeof(Step), cudaMemcpyHostToDevice, stream);
+        if (e != cudaSuccess) { static_forget_schedule(device); return BIGBIRD_ECUDA; }
+        static_remember_schedule(device, L->uid);
+    }
 
     const unsigned long long* kbits = nullptr;
     if (key_padding_mask) {
@@ -1113,10 +1419,24 @@ extern "C" int bigbird_attn_fwd_static(const void* q, const void* k, const void*
     p.nb = L->nb;
     p.total_work = p.BH * L->items_per_head;
     p.scale_log2 = scale * 1.4426950408889634f;
-    int grid = 2 * sd.sm_count;
-    if (grid > p.total_work) grid = p.total_work;
-    if (grid < 1) grid = 1;
+    const int grid = grid_size(sd.sm_count, p.total_work);
     attn_fwd_sm100_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tm_q, tm_k, tm_v, p);
     if (cudaGetLastError() != cudaSuccess) return BIGBIRD_ECUDA;
+    return BIGBIRD_OK;
+}
+
+extern "C" int bigbird_last_status_static(void* stream, int* status, int* detail) {
+    using namespace bigbird;
+    if (!status) return BIGBIRD_EINVAL;
+    int device = 0;
+    if (cudaGetDevice(&device) != cudaSuccess) return BIGBIRD_ECUDA;
+    if (device < 0 || device >= 64) return BIGBIRD_EUNSUPPORTED;
+    StaticDevice sd;
+    if (static_setup(device, &sd) != cudaSuccess) return BIGBIRD_ECUDA;
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return BIGBIRD_ECUDA;
+    int host[2] = {0, 0};                       // a stack buffer: nothing is allocated
+    if (cudaMemcpy(host, sd.base, sizeof(host), cudaMemcpyDeviceToHost) != cudaSuccess) return BIGBIRD_ECUDA;
+    *status = host[0];
+    if (detail) *detail = host[1];
     return BIGBIRD_OK;
 }

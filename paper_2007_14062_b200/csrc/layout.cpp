@@ -3,6 +3,7 @@
 #include "layout.h"
 
 #include <algorithm>
+#include <atomic>
 #include <new>
 
 #include "../../include/bigbird.h"
@@ -167,6 +168,9 @@ int build_layout_host(bigbird_layout* L, int chunk_steps) {
             L->items.push_back(it);
         }
     }
+    L->items_abs = L->items;
+    for (int h = 0; h < H; ++h)
+        for (int i = 0; i < L->items_per_head; ++i) L->items_abs[(size_t)h * L->items_per_head + i].step_begin += L->step_base[h];
     return BIGBIRD_OK;
 }
 
@@ -188,6 +192,8 @@ int bigbird_build_layout(int64_t N, int b, int w, int g, int r, uint64_t seed, i
     if (!L) return BIGBIRD_ENOMEM;
     L->N = N; L->b = b; L->w = w; L->g = g; L->r = r; L->H = H; L->mode = mode; L->seed = seed;
     L->nb = (int)nb64;
+    static std::atomic<uint64_t> next_uid{1};
+    L->uid = next_uid.fetch_add(1);
     int rc;
     try {
         rc = bigbird::build_layout_host(L, 0);

@@ -44,6 +44,7 @@ struct bigbird_layout {
     int64_t N;
     int b, w, g, r, H, mode;
     uint64_t seed;
+    uint64_t uid;                              // unique per handle for the life of the process, never 0
     int nb;
     // CSR over rows h*nb + j (the exported product)
     std::vector<int32_t> row_ptr;
@@ -53,7 +54,8 @@ struct bigbird_layout {
     int heavy_items_per_head = 0;   // leading items of each head that belong to global tiles
     int split_tiles_per_head = 0;   // global tiles cut into chunks (each needs a merge)
     int max_parts = 1;
-    std::vector<bigbird::Item> items;          // [H * items_per_head]
+    std::vector<bigbird::Item> items;          // [H * items_per_head], step_begin relative to the head's first step
+    std::vector<bigbird::Item> items_abs;      // the same with step_begin made absolute (what the kernel reads)
     std::vector<int32_t> step_base;            // [H] offset of the head's steps in `steps`
     std::vector<bigbird::Step> steps;
     std::vector<int32_t> split_tile_q;         // [split_tiles_per_head * 2] query blocks (qa, qb) of each split tile

@@ -34,6 +34,29 @@ def test_layout_sweep_bit_exact():
         L.close()
 
 
+def test_library_random_blocks_match_hand_worked_vectors():
+    """The library's own selection against the hand-worked vectors of tests/golden/random_blocks_seed0.txt
+    (App. D item 1 under the generator spec of bigbird.h), independently of the oracle."""
+    import os
+    path = os.path.join(os.path.dirname(__file__), "golden", "random_blocks_seed0.txt")
+    n = 0
+    for ln in open(path):
+        if not ln.strip() or ln.startswith("#"):
+            continue
+        lhs, rhs = ln.split(":")
+        nb, w, g, r, seed, h, j = (int(x) for x in lhs.split())
+        want = [int(x) for x in rhs.split()]
+        hw = (w - 1) // 2
+        window = [c for c in range(j - hw, j + hw + 1) if 0 <= c < nb]
+        L = bb.bigbird_build_layout(nb * 2, 2, w, g, r, seed, h + 1, bb.BIGBIRD_ITC)
+        rp, ci = L.export()
+        row = h * nb + j
+        assert list(ci[rp[row]:rp[row + 1]]) == sorted(set(window) | set(want)), ln
+        L.close()
+        n += 1
+    assert n >= 3
+
+
 @pytest.mark.parametrize("name", synth.ORDER)
 def test_layout_of_the_five_workloads_bit_exact(name):
     wl = synth.WORKLOADS[name]

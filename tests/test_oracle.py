@@ -43,6 +43,26 @@ def test_stream_key_separates_seed_head_block():
     assert O.stream_key(0, 0, 1) == 1
 
 
+def _random_block_vectors():
+    out = []
+    for ln in _golden_lines("random_blocks_seed0.txt"):
+        lhs, rhs = ln.split(":")
+        nb, w, g, r, seed, h, j = (int(x) for x in lhs.split())
+        out.append((nb, w, g, r, seed, h, j, [int(x) for x in rhs.split()]))
+    return out
+
+
+def test_random_blocks_hand_worked_vectors():
+    """App. D item 1 under the written generator spec: selections worked by hand from SplitMix64's
+    published outputs (derivation in the golden file).  A different bounded draw (z mod m), a shuffle
+    from the far end or a draw with replacement gives other blocks."""
+    vecs = _random_block_vectors()
+    assert len(vecs) >= 3
+    for nb, w, g, r, seed, h, j, want in vecs:
+        for b in (1, 4):
+            assert O.random_blocks(O.Graph(nb * b, b, w, g, r, seed, h + 1, O.ITC), h, j) == want
+
+
 # ----------------------------------------------------------------------------- block sets
 def _params():
     out = []
@@ -334,7 +354,7 @@ def test_attention_wrapper_slices_and_rows():
 
 
 def test_graph_rejects_bad_parameters():
-    for bad in [dict(N=10, b=4), dict(w=2), dict(g=99), dict(r=-1), dict(mode=3), dict(H=0)]:
+    for bad in [dict(N=10, b=4), dict(w=2), dict(g=99), dict(r=-1), dict(mode=3), dict(H=0), dict(seed=1 << 24), dict(seed=-1)]:
         kw = dict(N=16, b=4, w=3, g=2, r=1, seed=0, H=1, mode=0)
         kw.update(bad)
         with pytest.raises(ValueError):

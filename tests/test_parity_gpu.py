@@ -87,6 +87,7 @@ SMALL = [
     _small("bf16", 1, 1, 1, g=1, r=0),                          # a single block
     _small("bf16", 1, 2, 131, lengths="fixed:7000"),            # long sequence: the global tile is split along the keys
     _small("bf16", 2, 1, 100, g=3, r=2),                        # split global tiles, an unpaired global block
+    _small("bf16", 1, 1, 120, w=101, lengths="fixed:7000"),     # wide window: a sparse tile's key list spans two posted segments
     _small("fp32", 2, 2, 10, lengths="ragged:64:640"),
     _small("fp32", 1, 2, 7, mode=1, g=1, r=2),
 ]
@@ -171,7 +172,8 @@ def test_c2_base_itc_bf16_full_size():
     q, k, v = synth.make_qkv(wl)
     out, lse = _run(wl, q, k, v, None)
     assert np.isfinite(out).all() and np.isfinite(lse).all()
-    _compare(wl, q, k, v, None, out, lse, slices=_sample_slices(wl, 6) + [(0, 0), (wl.B - 1, wl.H - 1)])
+    # every (batch, head) slice, head-major so that the oracle builds each head's mask once
+    _compare(wl, q, k, v, None, out, lse, slices=[(bi, h) for h in range(wl.H) for bi in range(wl.B)])
 
 
 def test_c2_full_size_closed_forms():
@@ -200,7 +202,7 @@ def test_c3_etc_bf16_full_size():
     q, k, v = synth.make_qkv(wl)
     out, lse = _run(wl, q, k, v, None)
     assert np.isfinite(out).all() and np.isfinite(lse).all()
-    _compare(wl, q, k, v, None, out, lse, slices=_sample_slices(wl, 5) + [(0, 0)])
+    _compare(wl, q, k, v, None, out, lse, slices=[(bi, h) for h in range(wl.H) for bi in range(wl.B)])
 
 
 def test_c4_long_itc_bf16_full_size():
