@@ -56,15 +56,15 @@ constexpr int kStreams = 2;                // tile streams per CTA
 constexpr int kThreads = 512;
 constexpr int kWarpEpilogue = 8, kWarpProducer = 12, kWarpMma = 13, kWarpScheduler = 15;
 constexpr int kSoftmaxThreads = 128;
+// 512 threads x 128 registers fill the register file; no role needs more (the softmax threads hold one key block's
+// scores at a time), so the register split between roles stays even and nothing spills: a spill here costs a trip
+// to L2, since nearly all of the SM's L1 is configured as shared memory.
 #ifndef BB_REGS_SOFTMAX
 #define BB_REGS_SOFTMAX 184
 #define BB_REGS_EPILOGUE 80
 #define BB_REGS_LIGHT 64
 #endif
-constexpr int kRegsSoftmax = BB_REGS_SOFTMAX;          // registers per thread after setmaxnreg, by role
-constexpr int kRegsEpilogue = BB_REGS_EPILOGUE;
-constexpr int kRegsLight = BB_REGS_LIGHT;
-static_assert(kStreams * kRegsSoftmax + kRegsEpilogue + kRegsLight <= 512, "register file: 65536 = 128 threads x 512");
+constexpr int kRegsSoftmax = BB_REGS_SOFTMAX, kRegsEpilogue = BB_REGS_EPILOGUE, kRegsLight = BB_REGS_LIGHT;
 constexpr int kTmemCols = 512;
 constexpr int kStreamCols = kTmemCols / kStreams;
 constexpr int kColS = 0;                   // scores: kStepChunks x 64 fp32 columns
@@ -194,28 +194,27 @@ __device__ __forceinline__ bool mbar_test(unsigned long long* bar, unsigned pari
     return ok != 0;
 }
 
-// Bounded wait.  Returns false if the wait expired or another thread of the CTA already gave up.  The limit is
-// counted in SM clock cycles (a read of the cycle counter is cheap, unlike one of the global nanosecond timer)
-// and the counter is first read only after 64 failed tries.
-__device__ __forceinline__ bool mbar_wait_slow(unsigned long long* bar, unsigned parity, int* abort_flag, int* status, int code) {
-    long long t0 = 0;
-    for (unsigned it = 0;; ++it) {
+// Bounded wait, small enough to sit inline at every site (the kernel has to fit the SM's instruction cache of about
+// 32 KB: a loop with a clock read and its own give-up code per site did not).  Each try suspends the thread for up
+// to kTrySuspendNs; after kWaitTries failed tries (a few tenths of a second to two seconds, depending on how long
+// the hardware really keeps a thread suspended) the wait is abandoned.  Returns false then, or as soon as another
+// thread of the CTA has given up; the caller leaves its loop and calls give_up with the code of the wait.
+constexpr unsigned kTrySuspendNs = 1000;
+constexpr unsigned kWaitTries = 1500000;
+__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned parity, int* abort_flag) {
+#pragma unroll 1
+    for (unsigned it = 0; it < kWaitTries; ++it) {
         if (mbar_try(bar, parity)) return true;
-        if ((it & 63u) == 63u) {
-            if (*(volatile int*)abort_flag) return false;
-            const long long now = clock64();
-            if (it == 63u) t0 = now;
-            if (now - t0 > kWaitLimitCycles) {
-                if (atomicCAS(status, 0, BIGBIRD_ETIMEOUT) == 0) status[1] = code;
-                *(volatile int*)abort_flag = 1;
-                return false;
-            }
-        }
+        if (*(volatile int*)abort_flag) break;
     }
+    return false;
 }
-__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned parity, int* abort_flag, int* status, int code) {
-    if (__builtin_expect(mbar_try(bar, parity), 1)) return true;
-    return mbar_wait_slow(bar, parity, abort_flag, status, code);
+// Records BIGBIRD_ETIMEOUT and the code of the abandoned wait (the first one wins) and tells the rest of the CTA.
+__device__ __forceinline__ void give_up(int* abort_flag, int* status, int code) {
+    if (*(volatile int*)abort_flag == 0) {
+        if (atomicCAS(status, 0, BIGBIRD_ETIMEOUT) == 0) status[1] = code;
+        *(volatile int*)abort_flag = 1;
+    }
 }
 // The same bound for a role that polls: tick() is called whenever a round over the role's barriers found nothing
 // to do; it backs off (a polling warp that spins takes issue slots from the softmax warps of its sub-partition)
@@ -231,8 +230,7 @@ struct IdleClock {
             const long long now = clock64();
             if (n == 16u) t0 = now;
             else if (now - t0 > kWaitLimitCycles) {
-                if (atomicCAS(status, 0, BIGBIRD_ETIMEOUT) == 0) status[1] = code;
-                *(volatile int*)abort_flag = 1;
+                give_up(abort_flag, status, code);
                 return false;
             }
         }
@@ -394,18 +392,21 @@ __device__ __forceinline__ float row_max64(const float* s) {
 // Rare paths of the softmax threads.
 // -inf over the scores of the padded keys of one key block, in tensor memory.
 __device__ __forceinline__ void mask_scores(unsigned taddr, unsigned long long kb) {
-    float s[64];
-    tmem_ld64(taddr, s);
-    tmem_wait_ld();
+#pragma unroll 1
+    for (int h = 0; h < 2; ++h) {                   // 32 keys at a time (rolled: a rare path should not take up code space)
+        float s[32];
+        const unsigned bits = (unsigned)(kb >> (32 * h));
+        tmem_ld32(taddr + 32 * h, s);
+        tmem_wait_ld();
 #pragma unroll
-    for (int t = 0; t < 64; ++t) s[t] = ((kb >> t) & 1ull) ? s[t] : -INFINITY;
-    tmem_st32(taddr, reinterpret_cast<unsigned*>(s));
-    tmem_st32(taddr + 32, reinterpret_cast<unsigned*>(s + 32));
+        for (int t = 0; t < 32; ++t) s[t] = ((bits >> t) & 1u) ? s[t] : -INFINITY;
+        tmem_st32(taddr + 32 * h, reinterpret_cast<unsigned*>(s));
+    }
     tmem_wait_st();
 }
 // This thread's row of the output accumulator times alpha (the running maximum moved by more than the threshold).
 __device__ __forceinline__ void rescale_accumulator(unsigned taddr, float alpha) {
-#pragma unroll
+#pragma unroll 1
     for (int c = 0; c < 4; ++c) {
         float o[16];
         tmem_ld16(taddr + c * 16, o);
@@ -434,22 +435,18 @@ __device__ __forceinline__ int schedule_one(const KernelParams& p, SmemCtl* ctl,
     w = __shfl_sync(0xffffffffu, w, 0);
     if (w >= p.total_work) w = -1;
     // decode the work index: global-row tiles of every (batch, head) first, then the sparse tiles
-    int bh = 0, it = 0;
+    int bh = 0, it = 0, batch = 0;
     Item item{};
     if (w >= 0) {
         const int heavy_total = p.BH * p.heavy_per_head;
-        if (w < heavy_total) {
-            bh = w / p.heavy_per_head;
-            it = w - bh * p.heavy_per_head;
-        } else {
-            const int sparse = p.items_per_head - p.heavy_per_head;
-            const int w2 = w - heavy_total;
-            bh = w2 / sparse;
-            it = p.heavy_per_head + (w2 - bh * sparse);
-        }
-        item = p.items[(size_t)(bh % p.H) * p.items_per_head + it];
+        const bool heavy = w < heavy_total;
+        const unsigned per_head = heavy ? p.heavy_per_head : p.items_per_head - p.heavy_per_head;
+        const unsigned x = heavy ? w : w - heavy_total;
+        bh = (int)(x / per_head);                   // (one division for either kind of item: this code is kept small)
+        it = (int)(x - bh * per_head) + (heavy ? 0 : p.heavy_per_head);
+        batch = (int)((unsigned)bh / (unsigned)p.H);
+        item = p.items[(size_t)(bh - batch * p.H) * p.items_per_head + it];
     }
-    const int batch = bh / p.H;
     const unsigned long long qbits_a = w >= 0 ? key_bits(p, batch, item.qa) : 0ull;
     const unsigned long long qbits_b = w >= 0 ? key_bits(p, batch, item.qb) : 0ull;
     const bool tile_live = (qbits_a | qbits_b) != 0ull;      // a tile whose query rows are all padding is skipped
@@ -459,9 +456,10 @@ __device__ __forceinline__ int schedule_one(const KernelParams& p, SmemCtl* ctl,
     do {
         const unsigned ss = sched_n % kSchedSlots, sp = (sched_n / kSchedSlots) & 1u;
         // the first slot of an item is known to be free (the caller tested it); later segments of a long tile wait here
-        if (!mbar_wait(&sc->sched_empty[ss], sp ^ 1u, &ctl->abort_flag, p.status, 11)) return -2;
+        if (!mbar_wait(&sc->sched_empty[ss], sp ^ 1u, &ctl->abort_flag)) { give_up(&ctl->abort_flag, p.status, 11); return -2; }
         WorkSlot* slot = &sc->slot[ss];
         int count = 0;
+#pragma unroll 1
         while (i0 < n_raw && count <= kSegChunks - 32) {
             const int i = i0 + lane;
             ChunkEntry e{-1, 0, 0ull};
@@ -506,7 +504,7 @@ __device__ __forceinline__ int schedule_one(const KernelParams& p, SmemCtl* ctl,
 }
 
 __device__ __forceinline__ void scheduler_role(const KernelParams& p, SmemCtl* ctl, int lane) {
-    unsigned sched_n[kStreams] = {0, 0};
+    unsigned sched_n0 = 0, sched_n1 = 0;            // slots posted per stream (scalars: an indexed array would live in local memory)
     unsigned done = 0;                              // bit s: stream s has been told that there is no more work
     IdleClock idle;
     while (done != (1u << kStreams) - 1u) {
@@ -515,11 +513,11 @@ __device__ __forceinline__ void scheduler_role(const KernelParams& p, SmemCtl* c
         for (int s = 0; s < kStreams; ++s) {        // (not unrolled: one copy of the code)
             if ((done >> s) & 1u) continue;
             StreamCtl* sc = &ctl->st[s];
-            const unsigned ss = sched_n[s] % kSchedSlots, sp = (sched_n[s] / kSchedSlots) & 1u;
+            unsigned n = s == 0 ? sched_n0 : sched_n1;
+            const unsigned ss = n % kSchedSlots, sp = (n / kSchedSlots) & 1u;
             if (!__all_sync(0xffffffffu, mbar_test(&sc->sched_empty[ss], sp ^ 1u))) continue;
-            unsigned n = sched_n[s];
             const int w = schedule_one(p, ctl, sc, n, lane);
-            sched_n[s] = n;
+            if (s == 0) sched_n0 = n; else sched_n1 = n;
             if (w == -2) return;
             if (w < 0) done |= 1u << s;
             progress = true;
@@ -637,9 +635,10 @@ __device__ __forceinline__ void mma_role(const KernelParams& p, SmemCtl* ctl, co
     int* abort_flag = &ctl->abort_flag;
     unsigned ring_n = 0, q_n = 0, sched_n = 0, grp_n = 0, pv_n = 0, tile_n = 0;   // grp_n: steps whose Q K^T was issued; tile_n: tiles handed to the epilogue
     bool ok = true;
+    int fail = 0;                               // code of the wait that was abandoned, if any
     auto qk = [&](int cnt, unsigned qs) -> bool {   // S[:, 0 .. 64 cnt) = Q K^T with the K blocks of the next ring group
         const unsigned g = ring_n % kRingGroups, ph = (ring_n / kRingGroups) & 1u;
-        if (!mbar_wait(&sc->full[g], ph, abort_flag, p.status, 20)) return false;
+        if (!mbar_wait(&sc->full[g], ph, abort_flag)) { fail = 20; return false; }
         tc_fence_after();
         // the blocks of a group are adjacent: their 64 cnt rows form one K-major operand
         const unsigned long long q_desc = smem_desc_sw128(smem_u32(sr.smem + kStreamSmemQ + qs * 2 * kTileBytes));
@@ -658,16 +657,16 @@ __device__ __forceinline__ void mma_role(const KernelParams& p, SmemCtl* ctl, co
     int pend_n = 0, tile_steps = 0;
     auto pending_pv = [&]() -> bool {           // O (+)= sum_j P_j V_j with the V blocks of the next ring group
         if (pend_n == 0) return true;
-        if (!mbar_wait(&sc->p_full, pv_n & 1u, abort_flag, p.status, 22)) return false;
+        if (!mbar_wait(&sc->p_full, pv_n & 1u, abort_flag)) { fail = 22; return false; }
         // the epilogue must have taken the previous tile's accumulator before this tile's first P V overwrites it
-        if (pend_fresh && tile_n > 0 && !mbar_wait(&sc->o_free, (tile_n - 1) & 1u, abort_flag, p.status, 27)) return false;
+        if (pend_fresh && tile_n > 0 && !mbar_wait(&sc->o_free, (tile_n - 1) & 1u, abort_flag)) { fail = 27; return false; }
         const unsigned g = ring_n % kRingGroups, ph = (ring_n / kRingGroups) & 1u;
-        if (!mbar_wait(&sc->full[g], ph, abort_flag, p.status, 21)) return false;
+        if (!mbar_wait(&sc->full[g], ph, abort_flag)) { fail = 21; return false; }
         tc_fence_after();
         const unsigned long long v_desc = smem_desc_sw128(smem_u32(sr.smem + kStreamSmemRing + g * kGroupBytes));
-#pragma unroll
-        for (int j = 0; j < kStepChunks; ++j) {
-            if (j < pend_n) {
+#pragma unroll 1
+        for (int j = 0; j < pend_n; ++j) {
+            {
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk)  // 16 keys per MMA: 8 packed columns of P_j, two 8-row groups of V_j
                     mma_ts(sr.tmem + kColO, sr.tmem + kColP + 32 * j + kk * 8, v_desc + (unsigned long long)((j * kTileBytes + kk * 2048) >> 4), kIdescPV,
@@ -689,7 +688,7 @@ __device__ __forceinline__ void mma_role(const KernelParams& p, SmemCtl* ctl, co
     };
     while (ok) {
         const unsigned ss = sched_n % kSchedSlots, sp = (sched_n / kSchedSlots) & 1u;
-        if (!mbar_wait(&sc->sched_full[ss], sp, abort_flag, p.status, 23)) break;
+        if (!mbar_wait(&sc->sched_full[ss], sp, abort_flag)) { fail = 23; break; }
         const WorkSlot* slot = &sc->slot[ss];
         const int w = slot->w, flags = slot->flags, n = slot->n_chunks;
         if (w >= 0 && (flags & kSegLive) && (flags & kSegFirst)) {
@@ -708,12 +707,12 @@ __device__ __forceinline__ void mma_role(const KernelParams& p, SmemCtl* ctl, co
             if (work) {
                 // the softmax threads must have pulled the previous scores out of tensor memory
                 if (grp_n > 0) {
-                    ok = mbar_wait(&sc->s_free, (grp_n - 1) & 1u, abort_flag, p.status, 25);
-                    if (!ok) break;
+                    ok = mbar_wait(&sc->s_free, (grp_n - 1) & 1u, abort_flag);
+                    if (!ok) { fail = 25; break; }
                 }
                 if (q_unseen) {
-                    ok = mbar_wait(&sc->q_full[qs], qph, abort_flag, p.status, 24);
-                    if (!ok) break;
+                    ok = mbar_wait(&sc->q_full[qs], qph, abort_flag);
+                    if (!ok) { fail = 24; break; }
                     q_unseen = false;
                 }
                 tc_fence_after();
@@ -734,8 +733,8 @@ __device__ __forceinline__ void mma_role(const KernelParams& p, SmemCtl* ctl, co
         if (!ok) break;
         if (work && (flags & kSegLast)) {
             if (q_unseen) {                     // a tile without a live key block: its Q still has to land
-                ok = mbar_wait(&sc->q_full[qs], qph, abort_flag, p.status, 26);
-                if (!ok) break;
+                ok = mbar_wait(&sc->q_full[qs], qph, abort_flag);
+                if (!ok) { fail = 26; break; }
                 q_unseen = false;
             }
             tc_commit(&sc->q_empty[qs]);       // every Q K^T of the tile has been issued
@@ -745,6 +744,7 @@ __device__ __forceinline__ void mma_role(const KernelParams& p, SmemCtl* ctl, co
         ++sched_n;
         if (w < 0) break;
     }
+    if (fail) give_up(abort_flag, p.status, fail);
 }
 
 // ------------------------------------------------------------------------------------------------ softmax (one warpgroup per stream, one thread per row)
@@ -759,6 +759,7 @@ __device__ __forceinline__ void softmax_role(const KernelParams& p, SmemCtl* ctl
     const float sl2 = p.scale_log2;
     unsigned sched_n = 0, grp_n = 0, msg_n = 0;
     bool ok = true;
+    int fail = 0;                                   // code of the wait that was abandoned, if any
     float m_ref = -INFINITY, l_sum = 0.f;
     bool o_dirty = false;                           // has any P V been issued for this tile yet
     // exponentials of the 64 scores of one key block, packed in place: afterwards s[0..31] hold the bit
@@ -775,14 +776,14 @@ __device__ __forceinline__ void softmax_role(const KernelParams& p, SmemCtl* ctl
     };
     while (ok) {
         const unsigned ss = sched_n % kSchedSlots, sp = (sched_n / kSchedSlots) & 1u;
-        if (!mbar_wait(&sc->sched_full[ss], sp, abort_flag, p.status, 30)) break;
+        if (!mbar_wait(&sc->sched_full[ss], sp, abort_flag)) { fail = 30; break; }
         __syncwarp();
         const WorkSlot* slot = &sc->slot[ss];
         const int w = slot->w, flags = slot->flags, n = slot->n_chunks;
         if (w < 0) {                                // tell the epilogue that this stream is finished
             // (once it has taken the last tile: only then is it known to have read every earlier message, so that
             // the entry reused here is free)
-            if (msg_n > 0 && !mbar_wait(&sc->o_free, (msg_n - 1) & 1u, abort_flag, p.status, 36)) break;
+            if (msg_n > 0 && !mbar_wait(&sc->o_free, (msg_n - 1) & 1u, abort_flag)) { fail = 36; break; }
             EpiMsg* msg = &sc->epi[msg_n & 1u];
             if (row == 0) msg->kind = kEpiDone;
             mbar_arrive(&sc->epi_full[msg_n & 1u]);
@@ -801,32 +802,30 @@ __device__ __forceinline__ void softmax_role(const KernelParams& p, SmemCtl* ctl
             const int who0 = e[0].who, who1 = cnt > 1 ? e[1].who : kNoChunk;
             const bool mine0 = (who0 & kWhoMask) == kBothHalves || (who0 & kWhoMask) == my_who;
             const bool mine1 = (who1 & kWhoMask) == kBothHalves || (who1 & kWhoMask) == my_who;
-            ok = mbar_wait(&sc->s_full, grp_n & 1u, abort_flag, p.status, 31);
-            if (!ok) break;
+            ok = mbar_wait(&sc->s_full, grp_n & 1u, abort_flag);
+            if (!ok) { fail = 31; break; }
             __syncwarp();                           // lanes leave the wait one by one: back in step before the warp-wide loads
             tc_fence_after();
             // A key block with padded keys (rare: the one holding a sequence's end) gets -inf written over their
             // scores in tensor memory first, so that the common path below carries no masking code at all.
             if (__builtin_expect(((who0 | who1) & kHasPadding) != 0, 0)) {
-                if (mine0 && (who0 & kHasPadding)) mask_scores(lane_addr + kColS, e[0].kb);
-                if (mine1 && (who1 & kHasPadding)) mask_scores(lane_addr + kColS + 64, e[1].kb);
+#pragma unroll 1
+                for (int c = 0; c < cnt; ++c)
+                    if ((c == 0 ? mine0 : mine1) && (e[c].who & kHasPadding)) mask_scores(lane_addr + kColS + 64 * c, e[c].kb);
             }
-            // Two passes over the scores, each pulling them out of tensor memory: the row maximum first, then the
-            // exponentials one key block at a time in a loop that is not unrolled.  Reading twice is cheap; code that
-            // held all 128 scores in registers and was written out per key block was several times the size, and
-            // the kernel was bound by instruction fetch.
+            float s[128];
+            if (mine0) tmem_ld64(lane_addr + kColS, s);
+            if (mine1) tmem_ld64(lane_addr + kColS + 64, s + 64);
+            tmem_wait_ld();
+            // the score columns are free again: the next step's Q K^T may overwrite them
+            tc_fence_before();
+            mbar_arrive(&sc->s_free);
             float alpha = 1.f;
             bool rescale = false;
             if (mine0 || mine1) {
                 float m_loc = -INFINITY;
-#pragma unroll 1
-                for (int c = 0; c < cnt; ++c) {
-                    if (!((c == 0 ? mine0 : mine1))) continue;
-                    float s[64];
-                    tmem_ld64(lane_addr + kColS + 64 * c, s);
-                    tmem_wait_ld();
-                    m_loc = fmaxf(m_loc, row_max64(s));
-                }
+                if (mine0) m_loc = row_max64(s);
+                if (mine1) m_loc = fmaxf(m_loc, row_max64(s + 64));
                 const float m_cand = m_loc * sl2;
                 const bool need = m_cand > m_ref + kRescaleThreshold;        // true on the first step (m_ref = -inf)
                 rescale = __any_sync(0xffffffffu, need);
@@ -834,40 +833,25 @@ __device__ __forceinline__ void softmax_role(const KernelParams& p, SmemCtl* ctl
                     alpha = ex2(m_ref - m_cand);
                     m_ref = m_cand;
                 }
-            } else {
-                // nothing of this step is mine: the score columns are free as far as this thread is concerned
-                tc_fence_before();
-                mbar_arrive(&sc->s_free);
             }
+            // probabilities into registers first: the previous step's P V has this long to finish
             float sum0 = 0.f, sum1 = 0.f;
             const float neg_m = -m_ref;
-            const unsigned mine_bits = (mine0 ? 1u : 0u) | (mine1 ? 2u : 0u);
-#pragma unroll 1
-            for (int c = 0; c < cnt; ++c) {
-                const bool mine = (mine_bits >> c) & 1u;
-                float s[64];
-                if (mine) {
-                    tmem_ld64(lane_addr + kColS + 64 * c, s);
-                    tmem_wait_ld();
-                    if ((mine_bits >> (c + 1)) == 0u) {
-                        // my last scores of the step are in registers: the next step's Q K^T may overwrite the columns
-                        tc_fence_before();
-                        mbar_arrive(&sc->s_free);
-                    }
-                    exp_pack(s, neg_m, sum0, sum1);
-                }
-                if (c == 0) {
-                    // the previous step's P V must be complete before its probabilities are overwritten or O is touched
-                    if (grp_n > 0) {
-                        ok = mbar_wait(&sc->pv_done, (grp_n - 1) & 1u, abort_flag, p.status, 32);
-                        if (!ok) break;
-                        __syncwarp();
-                        tc_fence_after();
-                    }
-                    if (__builtin_expect(rescale && o_dirty, 0)) rescale_accumulator(lane_addr + kColO, alpha);
-                }
-                if (mine) tmem_st32(lane_addr + kColP + 32 * c, reinterpret_cast<unsigned*>(s));
-                else tmem_st32_zero(lane_addr + kColP + 32 * c);
+            if (mine0) exp_pack(s, neg_m, sum0, sum1);
+            if (mine1) exp_pack(s + 64, neg_m, sum0, sum1);
+            // the previous step's P V must be complete before its probabilities are overwritten or O is touched
+            if (grp_n > 0) {
+                ok = mbar_wait(&sc->pv_done, (grp_n - 1) & 1u, abort_flag);
+                if (!ok) { fail = 32; break; }
+                __syncwarp();
+                tc_fence_after();
+            }
+            if (__builtin_expect(rescale && o_dirty, 0)) rescale_accumulator(lane_addr + kColO, alpha);
+            if (mine0) tmem_st32(lane_addr + kColP, reinterpret_cast<unsigned*>(s));
+            else tmem_st32_zero(lane_addr + kColP);
+            if (cnt > 1) {
+                if (mine1) tmem_st32(lane_addr + kColP + 32, reinterpret_cast<unsigned*>(s + 64));
+                else tmem_st32_zero(lane_addr + kColP + 32);
             }
             if (!ok) break;
             l_sum = l_sum * alpha + (sum0 + sum1);
@@ -921,6 +905,7 @@ __device__ __forceinline__ void softmax_role(const KernelParams& p, SmemCtl* ctl
         mbar_arrive(&sc->sched_empty[ss]);
         ++sched_n;
     }
+    if (fail) give_up(abort_flag, p.status, fail);
 }
 
 // ------------------------------------------------------------------------------------------------ epilogue (one warpgroup, both streams)
@@ -934,13 +919,13 @@ __device__ __forceinline__ void epilogue_role(const KernelParams& p, SmemCtl* ct
     const bool lower = row >= kBlock;
     // per stream, packed so that the loop below is one copy of the code: bits 0..15 messages taken, 16..30 tiles
     // taken (only parities are used), bit 31 the stream is finished
-    unsigned state[kStreams] = {0u, 0u};
+    unsigned state0 = 0u, state1 = 0u;              // (scalars: an indexed array would live in local memory)
     IdleClock idle;
-    while (!((state[0] & state[1]) >> 31)) {
+    while (!((state0 & state1) >> 31)) {
         bool progress = false;
 #pragma unroll 1
         for (int s = 0; s < kStreams; ++s) {
-            const unsigned st = state[s];
+            const unsigned st = s == 0 ? state0 : state1;
             if (st >> 31) continue;
             StreamCtl* sc = &ctl->st[s];
             const unsigned msg_n = st & 0xffffu, tile_n = (st >> 16) & 0x7fffu;
@@ -948,11 +933,12 @@ __device__ __forceinline__ void epilogue_role(const KernelParams& p, SmemCtl* ct
             if (!__all_sync(0xffffffffu, mbar_test(&sc->epi_full[e], eph))) continue;
             progress = true;
             const EpiMsg* msg = &sc->epi[e];
-            if (msg->kind == kEpiDone) { state[s] = st | 0x80000000u; continue; }
-            state[s] = ((msg_n + 1u) & 0xffffu) | (((tile_n + 1u) & 0x7fffu) << 16);
+            const unsigned st_next = msg->kind == kEpiDone ? (st | 0x80000000u) : (((msg_n + 1u) & 0xffffu) | (((tile_n + 1u) & 0x7fffu) << 16));
+            if (s == 0) state0 = st_next; else state1 = st_next;
+            if (st_next >> 31) continue;
             const int bh = msg->bh, my_q = lower ? msg->qb : msg->qa, part_slot = msg->part_slot;
             const float inv = msg->inv[row];
-            if (!mbar_wait(&sc->o_done, tile_n & 1u, abort_flag, p.status, 40)) return;
+            if (!mbar_wait(&sc->o_done, tile_n & 1u, abort_flag)) { give_up(abort_flag, p.status, 40); return; }
             tc_fence_after();
             const unsigned lane_addr = tmem + s * kStreamCols + ((unsigned)(quad * 32) << 16);
             // the row's destination: the output tensor, or (raw fp32) the scratch of a split tile's part
@@ -988,7 +974,7 @@ __device__ __forceinline__ void epilogue_role(const KernelParams& p, SmemCtl* ct
         if (progress) idle.reset();
         else {
             // suspended on stream 0's next message for a short while; stream 1's is looked at again afterwards
-            const unsigned st0 = state[0];
+            const unsigned st0 = state0;
             if (!(st0 >> 31)) mbar_try_for(&ctl->st[0].epi_full[st0 & 1u], (st0 >> 1) & 1u, 300);
             else __nanosleep(300);
             if (!__all_sync(0xffffffffu, idle.tick(abort_flag, p.status, 41, 0))) return;
@@ -1117,7 +1103,7 @@ __global__ void wait_expiry_selftest_kernel(int* status) {
         mbar_init(&bar, 1);
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        mbar_wait(&bar, 0u, &abort_flag, status, 99);
+        if (!mbar_wait(&bar, 0u, &abort_flag)) give_up(&abort_flag, status, 99);
     }
 }
 
