@@ -41,6 +41,11 @@ Readings taken where the paper is silent (each is a deliberate choice):
   the attention graph itself does not depend on the mask.
 * lse is the natural log of the sum of exp(scaled, masked scores).
 
+* Backward pass (the paper trains through this op, Sec. 4 "Pretraining and MLM",
+  App. E.1, but prints no gradient formulas): the textbook derivatives of
+  Eq. (AT) under the same mask, written out in `attend_bwd`.  Padded QUERY rows
+  receive no gradient and give none (the library returns out = 0 for them).
+
 Everything is fp64.  Nothing here is blocked, fused or reordered.
 """
 from __future__ import annotations
@@ -232,4 +237,63 @@ def attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, gr: Graph,
         kv = None if key_padding_mask is None else (np.asarray(key_padding_mask[bi]) != 0)
         res[(bi, h)] = attend(np.asarray(q[bi, h], dtype=np.float64)[rws], k[bi, h], v[bi, h],
                               masks[h], kv, scale)
+    return res
+
+
+# --------------------------------------------------------------------------
+# Gradients of Eq. (AT) (the paper trains through the op; it prints no formulas).
+# --------------------------------------------------------------------------
+def attend_bwd(q_rows: np.ndarray, k: np.ndarray, v: np.ndarray, A_rows: np.ndarray,
+               key_valid: Optional[np.ndarray], scale: float, dout_rows: np.ndarray,
+               row_valid: Optional[np.ndarray] = None) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+    """Gradients of sum(out * dout) for a set of query rows of one (batch, head).
+
+    With S = scale q k^T restricted to the attended valid keys, P = softmax(S) and
+    out = P v:  dv = P^T dout,  dP = dout v^T,  dS = P o (dP - rowsum(dout o out)),
+    dq = scale dS k,  dk = scale dS^T q.  Rows with row_valid == False (padded
+    queries) and rows without any attended valid key contribute nothing and get
+    dq = 0.  Returns (dq fp64[R, D], dk fp64[N, D], dv fp64[N, D]); dk and dv
+    hold the contribution of these rows only.
+    """
+    q_rows = np.asarray(q_rows, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    v = np.asarray(v, dtype=np.float64)
+    dout_rows = np.asarray(dout_rows, dtype=np.float64)
+    S = scale * (q_rows @ k.T)
+    keep = A_rows if key_valid is None else (A_rows & np.asarray(key_valid, dtype=bool)[None, :])
+    if row_valid is not None:
+        keep = keep & np.asarray(row_valid, dtype=bool)[:, None]
+    S = np.where(keep, S, -np.inf)
+    m = S.max(axis=1)
+    safe_m = np.where(np.isfinite(m), m, 0.0)
+    E = np.exp(S - safe_m[:, None])
+    l = E.sum(axis=1)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        P = np.where(l[:, None] > 0, E / l[:, None], 0.0)
+    out = P @ v
+    dv = P.T @ dout_rows
+    dP = dout_rows @ v.T
+    delta = (dout_rows * out).sum(axis=1)
+    dS = P * (dP - delta[:, None])
+    dq = scale * (dS @ k)
+    dk = scale * (dS.T @ q_rows)
+    return dq, dk, dv
+
+
+def attention_bwd(q: np.ndarray, k: np.ndarray, v: np.ndarray, dout: np.ndarray, gr: Graph,
+                  key_padding_mask: Optional[np.ndarray], scale: float,
+                  slices: Optional[Sequence[Tuple[int, int]]] = None
+                  ) -> Dict[Tuple[int, int], Tuple[np.ndarray, np.ndarray, np.ndarray]]:
+    """BigBird attention gradients for [B, H, N, D] inputs: {(batch, head): (dq, dk, dv)} in fp64."""
+    B, H, N, D = q.shape
+    assert H == gr.H and N == gr.N
+    if slices is None:
+        slices = [(bi, h) for bi in range(B) for h in range(H)]
+    res = {}
+    masks: Dict[int, np.ndarray] = {}
+    for (bi, h) in slices:
+        if h not in masks:
+            masks = {h: build_mask(gr, h)}
+        kv = None if key_padding_mask is None else (np.asarray(key_padding_mask[bi]) != 0)
+        res[(bi, h)] = attend_bwd(q[bi, h], k[bi, h], v[bi, h], masks[h], kv, scale, dout[bi, h], row_valid=kv)
     return res

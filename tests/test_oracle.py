@@ -359,3 +359,78 @@ def test_graph_rejects_bad_parameters():
         kw.update(bad)
         with pytest.raises(ValueError):
             O.Graph(**kw)
+
+
+# ----------------------------------------------------------------------------- gradients
+def _loss(q, k, v, A, kv, scale, dout, rv=None):
+    out, _ = O.attend(q, k, v, A, kv, scale)
+    if rv is not None:
+        out = out * rv[:, None]
+    return float((out * dout).sum())
+
+
+@pytest.mark.parametrize("N,b,w,g,r,mode", [(12, 2, 3, 1, 1, O.ITC), (16, 1, 3, 2, 2, O.ITC), (14, 2, 3, 2, 0, O.ETC)])
+def test_gradients_match_central_differences_of_the_forward_oracle(N, b, w, g, r, mode):
+    """dq, dk, dv of `attend_bwd` against central finite differences of sum(out * dout) computed with the forward
+    oracle on the paper's toy sizes (App. D: 12 tokens, block 2; Fig. 1: token level), with padded keys and a
+    padded query row.  A dropped term, a wrong sign or a transposed operand shows up here."""
+    gr = O.Graph(N, b, w, g, r, 3, 1, mode)
+    rng = np.random.default_rng(N)
+    D = 4
+    q, k, v, dout = (rng.standard_normal((N, D)) for _ in range(4))
+    kv = np.ones(N, dtype=bool)
+    kv[-3:] = False
+    A = O.build_mask(gr, 0)
+    scale = 0.7
+    dq, dk, dv = O.attend_bwd(q, k, v, A, kv, scale, dout, row_valid=kv)
+    eps = 1e-6
+    for name, x, g_ in (("q", q, dq), ("k", k, dk), ("v", v, dv)):
+        num = np.zeros_like(x)
+        for idx in np.ndindex(*x.shape):
+            old = x[idx]
+            x[idx] = old + eps
+            fp = _loss(q, k, v, A, kv, scale, dout, kv.astype(float))
+            x[idx] = old - eps
+            fm = _loss(q, k, v, A, kv, scale, dout, kv.astype(float))
+            x[idx] = old
+            num[idx] = (fp - fm) / (2 * eps)
+        assert np.abs(num - g_).max() < 1e-7, name
+    assert (dq[~kv] == 0).all()                       # a padded query row gets no gradient
+    assert np.abs(dk[~kv]).max() == 0 and np.abs(dv[~kv]).max() == 0      # a padded key gets none either
+
+
+def test_gradients_on_the_complete_digraph_match_autograd_through_sdpa():
+    """Sec. 2: on the complete digraph Eq. (AT) is full attention, so the gradients must be those torch's
+    autograd computes through scaled_dot_product_attention in fp64."""
+    N, D = 24, 8
+    gr = O.Graph(N, 4, 2 * (N // 4) - 1, 0, 0, 0, 1, O.ITC)
+    A = O.build_mask(gr, 0)
+    assert A.all()
+    rng = np.random.default_rng(5)
+    q, k, v, dout = (rng.standard_normal((N, D)) for _ in range(4))
+    scale = 1.0 / math.sqrt(D)
+    dq, dk, dv = O.attend_bwd(q, k, v, A, None, scale, dout)
+    tq, tk, tv = (torch.tensor(x, dtype=torch.float64, requires_grad=True) for x in (q, k, v))
+    out = torch.nn.functional.scaled_dot_product_attention(tq[None, None], tk[None, None], tv[None, None], scale=scale)[0, 0]
+    (out * torch.tensor(dout)).sum().backward()
+    assert np.abs(tq.grad.numpy() - dq).max() < 1e-12
+    assert np.abs(tk.grad.numpy() - dk).max() < 1e-12
+    assert np.abs(tv.grad.numpy() - dv).max() < 1e-12
+
+
+def test_gradient_closed_forms_and_wrapper():
+    """Q == 0 makes every row uniform over its attended keys: dk == 0 and dv[key] = sum over the rows attending
+    it of dout[row] / (number of keys the row attends).  The wrapper loops (batch, head) slices over attend_bwd."""
+    gr = O.Graph(32, 4, 3, 2, 1, 1, 2, O.ITC)
+    rng = np.random.default_rng(9)
+    B, D = 2, 4
+    q = np.zeros((B, gr.H, gr.N, D))
+    k, v, dout = (rng.standard_normal((B, gr.H, gr.N, D)) for _ in range(3))
+    res = O.attention_bwd(q, k, v, dout, gr, None, 0.5)
+    for (bi, h), (dq, dk, dv) in res.items():
+        A = O.build_mask(gr, h).astype(np.float64)
+        W = A / A.sum(axis=1, keepdims=True)
+        assert np.abs(dk).max() < 1e-15
+        assert np.abs(dv - W.T @ dout[bi, h]).max() < 1e-13
+        want = O.attend_bwd(q[bi, h], k[bi, h], v[bi, h], O.build_mask(gr, h), None, 0.5, dout[bi, h])
+        assert all(np.array_equal(a, b) for a, b in zip((dq, dk, dv), want))
