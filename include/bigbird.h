@@ -82,6 +82,10 @@ BIGBIRD_API int bigbird_layout_nnz(const bigbird_layout* layout, int64_t* nnz);
  * col_idx: host int32[nnz].  Both caller-owned. */
 BIGBIRD_API int bigbird_layout_export(const bigbird_layout* layout, int32_t* row_ptr, int32_t* col_idx);
 
+/* The same graph by key block (what the gradients of K and V walk): row h * (N/b) + c lists, ascending, the query
+ * blocks that attend key block c.  col_ptr: host int32[H * N/b + 1]; row_idx: host int32[nnz].  Both caller-owned. */
+BIGBIRD_API int bigbird_layout_export_transposed(const bigbird_layout* layout, int32_t* col_ptr, int32_t* row_idx);
+
 /*
  * Introspection of the tile schedule derived from the lists (used by the tests; not needed to run attention).
  * The tensor-core kernel stacks two query blocks into one 2b-row tile (upper half, lower half) and walks a
@@ -134,6 +138,28 @@ BIGBIRD_API int bigbird_attn_fwd(const void* q, const void* k, const void* v, co
 BIGBIRD_API int bigbird_attn_fwd_simt(const void* q, const void* k, const void* v, const bigbird_layout* layout,
                           const uint8_t* key_padding_mask, void* out, float* lse,
                           int B, int H, int64_t N, int D, int b, float scale, int dtype, void* stream);
+
+/*
+ * bigbird_attn_bwd -- gradients of Eq. (AT) over the graph held by `layout` (the paper trains through this
+ * operation: Sec. 4 "Pretraining and MLM", App. E.1; it prints no gradient formulas, these are the derivatives of
+ * the softmax attention above).  Given dout = d loss / d out:
+ *
+ *     dv = P^T dout,   dS = P o (dout v^T - rowsum(dout o out)),   dq = scale dS k,   dk = scale dS^T q
+ *
+ * with P the attention probabilities, recomputed from q, k and the saved lse.
+ *
+ *   q, k, v, out, dout   device, [B, H, N, D] contiguous, one dtype (fp32 or bf16), 16-byte aligned; out and lse
+ *             are the results of bigbird_attn_fwd on the same q, k, v, layout, mask and scale
+ *   lse       device fp32 [B, H, N] (required)
+ *   dq, dk, dv  device, [B, H, N, D], same dtype; every element is written.  A padded QUERY row gets dq = 0 and gives
+ *             nothing to dk, dv; a padded key gets dk = dv = 0.
+ * Runs on CUDA cores in fp32 arithmetic for either dtype (D in {32, 64, 128}, any b): a first, correct path; there is
+ * no tensor-core gradient kernel yet.  Allocates nothing beyond the layout's device copy; only enqueues work.
+ * Errors: BIGBIRD_EINVAL, BIGBIRD_EUNSUPPORTED, BIGBIRD_ECUDA.
+ */
+BIGBIRD_API int bigbird_attn_bwd(const void* q, const void* k, const void* v, const void* out, const float* lse, const void* dout,
+                     const bigbird_layout* layout, const uint8_t* key_padding_mask, void* dq, void* dk, void* dv,
+                     int B, int H, int64_t N, int D, int b, float scale, int dtype, void* stream);
 
 /*
  * bigbird_attn_fwd_static -- bigbird_attn_fwd for callers that must not allocate device memory.  (The paper has

@@ -13,6 +13,7 @@ from .binding import (  # noqa: F401
     BIGBIRD_ITC,
     BigBirdError,
     Layout,
+    bigbird_attn_bwd,
     bigbird_attn_fwd,
     bigbird_attn_fwd_simt,
     bigbird_attn_fwd_static,

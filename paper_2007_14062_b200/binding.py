@@ -44,12 +44,14 @@ def lib() -> C.CDLL:
     L.bigbird_build_layout.argtypes = [i64, i32, i32, i32, i32, u64, i32, i32, C.POINTER(vp)]
     L.bigbird_layout_nnz.argtypes = [vp, C.POINTER(i64)]
     L.bigbird_layout_export.argtypes = [vp, vp, vp]
+    L.bigbird_layout_export_transposed.argtypes = [vp, vp, vp]
     L.bigbird_layout_schedule.argtypes = [vp, vp, vp, vp, vp]
     L.bigbird_layout_destroy.argtypes = [vp]
     fwd = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i64, i32, i32, f32, i32, vp]
     L.bigbird_attn_fwd.argtypes = fwd
     L.bigbird_attn_fwd_simt.argtypes = fwd
     L.bigbird_attn_fwd_static.argtypes = fwd
+    L.bigbird_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i64, i32, i32, f32, i32, vp]
     L.bigbird_last_status.argtypes = [vp, C.POINTER(i32), C.POINTER(i32)]
     L.bigbird_last_status_static.argtypes = [vp, C.POINTER(i32), C.POINTER(i32)]
     L.bigbird_last_cuda_error.argtypes = []
@@ -57,7 +59,7 @@ def lib() -> C.CDLL:
     L.bigbird_last_launch_count.argtypes = []
     L.bigbird_strerror.argtypes = [i32]
     L.bigbird_strerror.restype = C.c_char_p
-    for name in ("bigbird_build_layout", "bigbird_layout_nnz", "bigbird_layout_export", "bigbird_layout_schedule",
+    for name in ("bigbird_build_layout", "bigbird_layout_nnz", "bigbird_layout_export", "bigbird_layout_export_transposed", "bigbird_layout_schedule", "bigbird_attn_bwd",
                  "bigbird_layout_destroy", "bigbird_attn_fwd", "bigbird_attn_fwd_simt", "bigbird_attn_fwd_static", "bigbird_last_status", "bigbird_last_status_static",
                  "bigbird_last_cuda_error", "bigbird_last_launch_count", "bigbird_selftest_wait_expiry"):
         getattr(L, name).restype = i32
@@ -91,6 +93,14 @@ class Layout:
         _check(lib().bigbird_layout_export(self.handle, row_ptr.ctypes.data, col_idx.ctypes.data),
                "bigbird_layout_export")
         return row_ptr, col_idx[: self.nnz]
+
+    def export_transposed(self) -> Tuple[np.ndarray, np.ndarray]:
+        """The graph by key block: (col_ptr int32[H*nb+1], row_idx int32[nnz]) over rows h*nb + c."""
+        col_ptr = np.empty(self.H * self.nb + 1, dtype=np.int32)
+        row_idx = np.empty(max(self.nnz, 1), dtype=np.int32)
+        _check(lib().bigbird_layout_export_transposed(self.handle, col_ptr.ctypes.data, row_idx.ctypes.data),
+               "bigbird_layout_export_transposed")
+        return col_ptr, row_idx[: self.nnz]
 
     def schedule(self):
         """(sizes, items int32[H*ipH, 8], step_base int32[H], steps int32[S, 2]) of the tile schedule."""
@@ -164,6 +174,34 @@ def bigbird_attn_fwd_static(q, k, v, layout: Layout, key_padding_mask, out, lse,
     inside the loaded module.  bf16, D == 64, b == 64 only; BigBirdError(-6) if the problem exceeds the array.
     Calls on one device must not overlap on the GPU; make the first call on a device outside stream capture."""
     _fwd("bigbird_attn_fwd_static", q, k, v, layout, key_padding_mask, out, lse, scale, stream)
+
+
+def bigbird_attn_bwd(q, k, v, out, lse, dout, layout: Layout, key_padding_mask, dq, dk, dv, scale: float,
+                     stream: Optional[int] = None) -> None:
+    """Enqueues the gradient kernels: dq, dk, dv from dout and the forward pass's out and lse."""
+    ts = (q, k, v, out, dout, dq, dk, dv)
+    if not all(t.is_cuda for t in ts):
+        raise ValueError("all tensors must be CUDA tensors (there is no CPU path)")
+    for t in ts:
+        if not t.is_contiguous() or t.shape != q.shape or t.dtype != q.dtype:
+            raise ValueError("q, k, v, out, dout, dq, dk, dv must be contiguous [B, H, N, D] tensors of one dtype")
+    B, H, N, D = q.shape
+    dtype = {torch.float32: BIGBIRD_FP32, torch.bfloat16: BIGBIRD_BF16}.get(q.dtype)
+    if dtype is None:
+        raise ValueError("dtype must be float32 or bfloat16")
+    if lse.dtype != torch.float32 or tuple(lse.shape) != (B, H, N) or not lse.is_cuda or not lse.is_contiguous():
+        raise ValueError("lse must be a contiguous CUDA float32 [B, H, N] tensor")
+    if key_padding_mask is not None:
+        if key_padding_mask.dtype != torch.uint8 or tuple(key_padding_mask.shape) != (B, N) or \
+                not key_padding_mask.is_cuda or not key_padding_mask.is_contiguous():
+            raise ValueError("key_padding_mask must be a contiguous CUDA uint8 [B, N] tensor")
+    if stream is None:
+        stream = torch.cuda.current_stream(q.device).cuda_stream
+    with torch.cuda.device(q.device):
+        code = lib().bigbird_attn_bwd(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), _ptr(dout), layout.handle,
+                                      _ptr(key_padding_mask), _ptr(dq), _ptr(dk), _ptr(dv), B, H, N, D, layout.b,
+                                      float(scale), dtype, C.c_void_p(stream))
+    _check(code, "bigbird_attn_bwd")
 
 
 def bigbird_last_status(stream: Optional[int] = None) -> Tuple[int, int]:

@@ -9,7 +9,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libbigbird.so")
-SOURCES = ["layout.cpp", "api.cu", "attn_fwd_simt.cu", "attn_fwd_sm100.cu"]
+SOURCES = ["layout.cpp", "api.cu", "attn_fwd_simt.cu", "attn_bwd_simt.cu", "attn_fwd_sm100.cu"]
 HEADERS = ["layout.h", "kernels.h", os.path.join("..", "..", "include", "bigbird.h")]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

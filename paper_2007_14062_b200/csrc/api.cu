@@ -52,6 +52,8 @@ cudaError_t upload(T** dst, const void* src, size_t count) {
 void free_device_layout(DeviceLayout& d) {
     cudaFree(d.row_ptr);
     cudaFree(d.col_idx);
+    cudaFree(d.col_ptr);
+    cudaFree(d.row_idx);
     cudaFree(d.items);
     cudaFree(d.steps);
     cudaFree(d.split_tile_q);
@@ -71,6 +73,8 @@ int get_device_layout(const bigbird_layout* L, int device, DeviceLayout* out) {
         }
         cudaError_t e = upload(&d.row_ptr, L->row_ptr.data(), L->row_ptr.size());
         if (e == cudaSuccess) e = upload(&d.col_idx, L->col_idx.data(), L->col_idx.size());
+        if (e == cudaSuccess) e = upload(&d.col_ptr, L->col_ptr.data(), L->col_ptr.size());
+        if (e == cudaSuccess) e = upload(&d.row_idx, L->row_idx.data(), L->row_idx.size());
         if (e == cudaSuccess) e = upload(&d.items, L->items_abs.data(), L->items_abs.size());
         if (e == cudaSuccess) e = upload(&d.steps, L->steps.data(), L->steps.size());
         if (e == cudaSuccess) e = upload(&d.split_tile_q, L->split_tile_q.data(), L->split_tile_q.size());
@@ -139,6 +143,29 @@ int bigbird_attn_fwd_simt(const void* q, const void* k, const void* v, const big
                           const uint8_t* key_padding_mask, void* out, float* lse, int B, int H, int64_t N,
                           int D, int b, float scale, int dtype, void* stream) {
     return bigbird::fwd(true, q, k, v, layout, key_padding_mask, out, lse, B, H, N, D, b, scale, dtype, stream);
+}
+
+int bigbird_attn_bwd(const void* q, const void* k, const void* v, const void* out, const float* lse, const void* dout,
+                     const bigbird_layout* layout, const uint8_t* key_padding_mask, void* dq, void* dk, void* dv,
+                     int B, int H, int64_t N, int D, int b, float scale, int dtype, void* stream) {
+    using namespace bigbird;
+    t_last_launches = 0;
+    int rc = check_common(q, k, v, layout, dq, B, H, N, D, b, dtype);
+    if (rc != BIGBIRD_OK) return rc;
+    if (!out || !lse || !dout || !dk || !dv) return BIGBIRD_EINVAL;
+    if ((((uintptr_t)out) | ((uintptr_t)dout) | ((uintptr_t)dk) | ((uintptr_t)dv)) & 15) return BIGBIRD_EINVAL;
+    if (D != 32 && D != 64 && D != 128) return BIGBIRD_EUNSUPPORTED;
+    if ((int64_t)B * H > 65535) return BIGBIRD_EUNSUPPORTED;
+    if (!(scale > 0.f) || !(scale < INFINITY)) return BIGBIRD_EINVAL;
+    int device = 0;
+    cudaError_t e = cudaGetDevice(&device);
+    if (e != cudaSuccess) return cuda_fail(e);
+    DeviceLayout dl;
+    rc = get_device_layout(layout, device, &dl);
+    if (rc != BIGBIRD_OK) return rc;
+    BwdArgs a{q, k, v, out, lse, dout, key_padding_mask, dq, dk, dv, B, H, D, b, layout->nb, N, scale, dtype, (cudaStream_t)stream};
+    e = launch_attn_bwd_simt(a, dl, &t_last_launches);
+    return e == cudaSuccess ? BIGBIRD_OK : cuda_fail(e);
 }
 
 int bigbird_layout_destroy(bigbird_layout* L) {

@@ -87,6 +87,22 @@ int build_layout_host(bigbird_layout* L, int chunk_steps) {
         }
     }
 
+    // ---- the graph by key block (what the gradients of K and V walk) ----------------------------
+    L->col_ptr.assign((size_t)H * nb + 1, 0);
+    L->row_idx.assign(L->col_idx.size(), 0);
+    for (int h = 0; h < H; ++h)
+        for (int j = 0; j < nb; ++j)
+            for (int32_t e = L->row_ptr[(size_t)h * nb + j]; e < L->row_ptr[(size_t)h * nb + j + 1]; ++e)
+                ++L->col_ptr[(size_t)h * nb + L->col_idx[e] + 1];
+    for (size_t i = 0; i < (size_t)H * nb; ++i) L->col_ptr[i + 1] += L->col_ptr[i];
+    {
+        std::vector<int32_t> fill(L->col_ptr.begin(), L->col_ptr.end() - 1);
+        for (int h = 0; h < H; ++h)
+            for (int j = 0; j < nb; ++j)                                     // ascending j: each list comes out sorted
+                for (int32_t e = L->row_ptr[(size_t)h * nb + j]; e < L->row_ptr[(size_t)h * nb + j + 1]; ++e)
+                    L->row_idx[fill[(size_t)h * nb + L->col_idx[e]]++] = j;
+    }
+
     // ---- tile schedule ----------------------------------------------------------------------------
     // Query blocks are stacked two by two into 2b-row tiles: the global blocks among themselves (every key
     // block is attended by both halves), the others in ascending order.  A step is one key block together
@@ -215,6 +231,13 @@ int bigbird_layout_export(const bigbird_layout* L, int32_t* row_ptr, int32_t* co
     if (!L || !row_ptr || !col_idx) return BIGBIRD_EINVAL;
     std::copy(L->row_ptr.begin(), L->row_ptr.end(), row_ptr);
     std::copy(L->col_idx.begin(), L->col_idx.end(), col_idx);
+    return BIGBIRD_OK;
+}
+
+int bigbird_layout_export_transposed(const bigbird_layout* L, int32_t* col_ptr, int32_t* row_idx) {
+    if (!L || !col_ptr || !row_idx) return BIGBIRD_EINVAL;
+    std::copy(L->col_ptr.begin(), L->col_ptr.end(), col_ptr);
+    std::copy(L->row_idx.begin(), L->row_idx.end(), row_idx);
     return BIGBIRD_OK;
 }
 

@@ -33,6 +33,8 @@ struct DeviceLayout {
     int device = -1;
     int32_t* row_ptr = nullptr;
     int32_t* col_idx = nullptr;
+    int32_t* col_ptr = nullptr;
+    int32_t* row_idx = nullptr;
     Item* items = nullptr;
     Step* steps = nullptr;
     int32_t* split_tile_q = nullptr;   // [split_tiles_per_head * 2]
@@ -49,6 +51,9 @@ struct bigbird_layout {
     // CSR over rows h*nb + j (the exported product)
     std::vector<int32_t> row_ptr;
     std::vector<int32_t> col_idx;
+    // the same graph by key block: rows h*nb + c list, ascending, the query blocks that attend key block c
+    std::vector<int32_t> col_ptr;
+    std::vector<int32_t> row_idx;
     // tile schedule: per head the same number of items, heavy (global) items first
     int items_per_head = 0;
     int heavy_items_per_head = 0;   // leading items of each head that belong to global tiles

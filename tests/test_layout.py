@@ -71,6 +71,25 @@ def test_layout_of_the_five_workloads_bit_exact(name):
     assert (per_head == want).all()
 
 
+def test_transposed_lists_are_the_transpose_of_the_oracle_mask():
+    """Row (h, c) of the transposed export lists, ascending, the query blocks whose oracle mask attends key block c."""
+    for cfg in [(512, 64, 3, 2, 3, 0, 2, 0), (4224, 64, 3, 2, 0, 2, 2, 1), (13 * 4, 4, 5, 3, 2, 5, 3, 0), (6, 1, 3, 6, 0, 0, 1, 1),
+                (7 * 2, 2, 3, 0, 6, 1, 2, 0)]:
+        N, b, w, g, r, seed, H, mode = cfg
+        nb = N // b
+        L = bb.bigbird_build_layout(*cfg)
+        cp, ri = L.export_transposed()
+        assert cp.dtype == np.int32 and ri.dtype == np.int32 and cp[0] == 0 and cp[-1] == L.nnz
+        gr = O.Graph(N, b, w, g, r, seed, H, mode)
+        first = np.arange(nb) * b
+        for h in range(H):
+            A = O.mask_rows(gr, h, first)[:, first]                  # block-level adjacency [query block, key block]
+            for c in range(nb):
+                got = ri[cp[h * nb + c]:cp[h * nb + c + 1]]
+                assert list(got) == list(np.nonzero(A[:, c])[0]), (cfg, h, c)
+        L.close()
+
+
 def test_window_choice_is_moot_for_the_five_workloads():
     """With w=3 a circular window would only add blocks that are global anyway (first/last rows in ITC,
     block 0 in ETC), so clipped and circular windows give the same graph on all five workloads."""
