@@ -127,7 +127,8 @@ def test_closed_forms_on_gpu(impl, dtype):
     kpm = synth.key_padding_mask(wl)
     out, _ = _run(wl, q, k, torch.ones_like(v), kpm, impl)
     valid = kpm[0].numpy() != 0
-    assert np.abs(out[0][:, valid] - 1).max() <= (1e-6 if dtype == "fp32" else 2 ** -8)
+    # (fp32: numerator and denominator are the same sum taken in two orders; a few dozen fp32 roundings apart)
+    assert np.abs(out[0][:, valid] - 1).max() <= (4e-6 if dtype == "fp32" else 2 ** -8)
     out, lse = _run(wl, torch.zeros_like(q), k, v, kpm, impl)
     gr = _graph(wl)
     for h in range(wl.H):
