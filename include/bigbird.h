@@ -40,7 +40,9 @@ enum {
     BIGBIRD_ECUDA = -3,         /* a CUDA call failed; see bigbird_last_cuda_error() */
     BIGBIRD_ETIMEOUT = -4,      /* a bounded wait inside a kernel expired (reported by bigbird_last_status) */
     BIGBIRD_ENOMEM = -5,
-    BIGBIRD_ELIMIT = -6         /* the problem exceeds the fixed scratch of bigbird_attn_fwd_static */
+    BIGBIRD_ELIMIT = -6,        /* the problem exceeds the fixed scratch of bigbird_attn_fwd_static */
+    BIGBIRD_EINTERNAL = -7      /* a checked build (compiled with BB_DEBUG) found an index out of range inside a kernel; reported by
+                                   bigbird_last_status like BIGBIRD_ETIMEOUT, with the code of the check; the kernel skips the access */
 };
 
 enum { BIGBIRD_ITC = 0, BIGBIRD_ETC = 1 };

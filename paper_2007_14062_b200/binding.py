@@ -12,7 +12,8 @@ BIGBIRD_ITC, BIGBIRD_ETC = 0, 1
 BIGBIRD_FP32, BIGBIRD_BF16 = 0, 1
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "libbigbird.so")
+# BIGBIRD_LIB selects another build of the same library (the checked build libbigbird_debug.so, say)
+_LIB_PATH = os.environ.get("BIGBIRD_LIB") or os.path.join(_HERE, "libbigbird.so")
 _lib: Optional[C.CDLL] = None
 
 

@@ -131,7 +131,6 @@ attn_fwd_simt_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* 
 #pragma unroll
         for (int kk = 0; kk < KC; ++kk) {
             const float p = sp[rloc][kk];
-#pragma unroll
             if constexpr (DL >= 2) {
 #pragma unroll
                 for (int i = 0; i < DL; i += 2) {

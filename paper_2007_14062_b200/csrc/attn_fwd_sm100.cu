@@ -12,8 +12,9 @@
 //     tensor pipe full where one thread's issue rate would not (a 64-wide P V instruction takes the pipe less
 //     time than one thread needs to issue the next), and the two softmax warpgroups fill each other's gaps on
 //     the special-function unit.
-//   * A producer thread fetches Q once per tile and the K and V blocks with TMA (128-byte swizzle) straight
-//     from the [B, H, N, D] tensors into the stream's ring: nothing is gathered or packed in HBM.
+//   * Four lanes of a producer warp (per stream one for Q and K, one for V) fetch Q once per tile and the K and V
+//     blocks with TMA (128-byte swizzle) straight from the [B, H, N, D] tensors into the stream's ring: nothing is
+//     gathered or packed in HBM.
 //   * Key blocks are processed two at a time (one "step").  Their K tiles land in adjacent ring slots, so that
 //     S = Q K^T of a step is one N = 128 tcgen05.mma per 16 head dimensions.  O += P V follows with P read
 //     from tensor memory.
@@ -172,8 +173,9 @@ __device__ __forceinline__ unsigned long long global_ns() {
     return t;
 }
 
-// One try with a limit on the time the thread stays suspended (nanoseconds): what a role that watches several
-// barriers sleeps on between rounds, so that it neither spins nor oversleeps the one it is suspended on.
+// One try with a time hint.  On this part a failing try with a hint keeps the thread suspended for about 4 us
+// whatever the hint says (measured), and wakes early when the phase completes: a role that watches two barriers uses
+// it to sleep on one of them between rounds instead of spinning.
 __device__ __forceinline__ bool mbar_try_for(unsigned long long* bar, unsigned parity, unsigned ns) {
     unsigned ok;
     asm volatile(
@@ -194,12 +196,11 @@ __device__ __forceinline__ bool mbar_test(unsigned long long* bar, unsigned pari
     return ok != 0;
 }
 
-// Bounded wait, small enough to sit inline at every site (the kernel has to fit the SM's instruction cache of about
-// 32 KB: a loop with a clock read and its own give-up code per site did not).  Each try suspends the thread for up
-// to kTrySuspendNs; after kWaitTries failed tries (a few tenths of a second to two seconds, depending on how long
-// the hardware really keeps a thread suspended) the wait is abandoned.  Returns false then, or as soon as another
+// Bounded wait, small enough to sit inline at every site (the kernel's hot code has to fit the SM's instruction
+// cache, measured at between 32 and 48 KB: a loop with a clock read and its own give-up code per site did not).  A
+// failing try keeps the thread suspended for about 1.4 us on this part (measured); after kWaitTries of them, about
+// two seconds, the wait is abandoned.  Returns false then, or as soon as another
 // thread of the CTA has given up; the caller leaves its loop and calls give_up with the code of the wait.
-constexpr unsigned kTrySuspendNs = 1000;
 constexpr unsigned kWaitTries = 1500000;
 __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned parity, int* abort_flag) {
 #pragma unroll 1
@@ -216,6 +217,23 @@ __device__ __forceinline__ void give_up(int* abort_flag, int* status, int code) 
         *(volatile int*)abort_flag = 1;
     }
 }
+// Checked build (-DBB_DEBUG): indices that come out of the schedule are tested against their ranges before they are
+// used as addresses; a failing check records BIGBIRD_EINTERNAL with its code, tells the CTA to stop, and the access
+// is skipped.  Nothing traps.  (The memory checker is not available where this library is developed; small cases
+// against the oracle and this build stand in for it.)
+#ifdef BB_DEBUG
+__device__ __forceinline__ bool debug_check(bool good, int* abort_flag, int* status, int code) {
+    if (!good && *(volatile int*)abort_flag == 0) {
+        if (atomicCAS(status, 0, BIGBIRD_EINTERNAL) == 0) status[1] = code;
+        *(volatile int*)abort_flag = 1;
+    }
+    return good;
+}
+#define BB_CHECK(cond, code) debug_check((cond), &ctl->abort_flag, p.status, (code))
+#else
+#define BB_CHECK(cond, code) true
+#endif
+
 // The same bound for a role that polls: tick() is called whenever a round over the role's barriers found nothing
 // to do; it backs off (a polling warp that spins takes issue slots from the softmax warps of its sub-partition)
 // and returns false once the CTA has given up or the idle time exceeds the limit.
@@ -332,13 +350,6 @@ __device__ __forceinline__ void tmem_st32_zero(unsigned taddr) {
         "%0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0};"
         ::"r"(z), "r"(taddr) : "memory");
 }
-__device__ __forceinline__ void tmem_st16_zero(unsigned taddr) {
-    const unsigned z = 0;
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%1], "
-        "{%0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0, %0};"
-        ::"r"(z), "r"(taddr) : "memory");
-}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -445,7 +456,9 @@ __device__ __forceinline__ int schedule_one(const KernelParams& p, SmemCtl* ctl,
         bh = (int)(x / per_head);                   // (one division for either kind of item: this code is kept small)
         it = (int)(x - bh * per_head) + (heavy ? 0 : p.heavy_per_head);
         batch = (int)((unsigned)bh / (unsigned)p.H);
-        item = p.items[(size_t)(bh - batch * p.H) * p.items_per_head + it];
+        if (BB_CHECK(bh >= 0 && bh < p.BH && it >= 0 && it < p.items_per_head, 71)) item = p.items[(size_t)(bh - batch * p.H) * p.items_per_head + it];
+        else w = -1;
+        if (!BB_CHECK(item.step_count >= 0 && item.step_begin >= 0 && item.qa >= 0 && item.qa < p.nb && item.qb < p.nb, 72)) w = -1;
     }
     const unsigned long long qbits_a = w >= 0 ? key_bits(p, batch, item.qa) : 0ull;
     const unsigned long long qbits_b = w >= 0 ? key_bits(p, batch, item.qb) : 0ull;
@@ -473,9 +486,7 @@ __device__ __forceinline__ int schedule_one(const KernelParams& p, SmemCtl* ctl,
                 e.kb = key_bits(p, batch, s.c);
                 e.who = ((ua && ub) ? kBothHalves : (ua ? kUpperHalf : kLowerHalf)) | (e.kb != ~0ull ? kHasPadding : 0);
                 alive = e.kb != 0ull && (ua || ub);
-#ifdef BB_DEBUG
-                if (s.c < 0 || s.c >= p.nb) { debug_fail(ctl, p.status, 70); alive = false; }
-#endif
+                if (!BB_CHECK(s.c >= 0 && s.c < p.nb && (unsigned)s.who <= (unsigned)kLowerHalf, 70)) alive = false;
             }
             const unsigned bal = __ballot_sync(0xffffffffu, alive);
             if (alive) slot->chunks[count + __popc(bal & lt_mask)] = e;
@@ -527,105 +538,56 @@ __device__ __forceinline__ void scheduler_role(const KernelParams& p, SmemCtl* c
     }
 }
 
-// ------------------------------------------------------------------------------------------------ TMA producer (one thread per stream)
-// Ring order of a stream = the order in which its MMA thread consumes groups: K of step i, then V of step i-1.
-struct ProducerState {
-    unsigned ring_n = 0, q_n = 0, sched_n = 0;
-    int op = 0;                    // what the stream needs next (kOp*)
-    int w = 0, bh = 0, n = 0, i = 0;
-    int cur_n = 0, cur_c0 = 0, cur_c1 = 0;
-    int pend_n = 0, pend_bh = 0, pend_c0 = 0, pend_c1 = 0;
-};
-enum { kOpSlot = 0, kOpQ, kOpK, kOpV, kOpRelease, kOpFinalV, kOpDone };
-
-__device__ __forceinline__ void load_group(const KernelParams& p, const StreamRef& sr, const CUtensorMap* tm, unsigned g, int bh, int c0, int c1, int cnt) {
-    StreamCtl* sc = sr.sc;
-    mbar_expect_tx(&sc->full[g], cnt * kTileBytes);
-    tma_load_tile(sr.smem + kStreamSmemRing + g * kGroupBytes, tm, (bh * p.nb + c0) * kBlock, &sc->full[g]);
-    if (cnt > 1) tma_load_tile(sr.smem + kStreamSmemRing + g * kGroupBytes + kTileBytes, tm, (bh * p.nb + c1) * kBlock, &sc->full[g]);
-}
-
-// One non-blocking attempt to move the stream's loads forward.  Returns whether anything was done.
-__device__ __forceinline__ bool producer_advance(const KernelParams& p, const StreamRef& sr, ProducerState& st, const CUtensorMap* tm_q,
-                                                 const CUtensorMap* tm_k, const CUtensorMap* tm_v) {
-    StreamCtl* sc = sr.sc;
-    const unsigned ss = st.sched_n % kSchedSlots, sp = (st.sched_n / kSchedSlots) & 1u;
-    const WorkSlot* slot = &sc->slot[ss];
-    const unsigned g = st.ring_n % kRingGroups, gph = (st.ring_n / kRingGroups) & 1u;
-    switch (st.op) {
-        case kOpSlot: {
-            if (!mbar_test(&sc->sched_full[ss], sp)) return false;
-            st.w = slot->w;
-            st.bh = slot->bh;
-            st.n = slot->n_chunks;
-            st.i = 0;
-            const int flags = slot->flags;
-            if (st.w >= 0 && (flags & kSegLive)) st.op = (flags & kSegFirst) ? kOpQ : (st.n > 0 ? kOpK : kOpRelease);
-            else st.op = kOpRelease;
-            return true;
-        }
-        case kOpQ: {
-            const unsigned qs = st.q_n & 1u;
-            if (!mbar_test(&sc->q_empty[qs], ((st.q_n >> 1) & 1u) ^ 1u)) return false;
-            const int qa = slot->qa, qb = slot->qb;
-            mbar_expect_tx(&sc->q_full[qs], qb >= 0 ? 2 * kTileBytes : kTileBytes);
-            tma_load_tile(sr.smem + kStreamSmemQ + qs * 2 * kTileBytes, tm_q, (st.bh * p.nb + qa) * kBlock, &sc->q_full[qs]);
-            if (qb >= 0) tma_load_tile(sr.smem + kStreamSmemQ + qs * 2 * kTileBytes + kTileBytes, tm_q, (st.bh * p.nb + qb) * kBlock, &sc->q_full[qs]);
-            ++st.q_n;
-            st.op = st.n > 0 ? kOpK : kOpRelease;
-            return true;
-        }
-        case kOpK: {
-            if (!mbar_test(&sc->empty[g], gph ^ 1u)) return false;
-            st.cur_n = min(kStepChunks, st.n - st.i);
-            st.cur_c0 = slot->chunks[st.i].c;
-            st.cur_c1 = st.cur_n > 1 ? slot->chunks[st.i + 1].c : 0;
-            load_group(p, sr, tm_k, g, st.bh, st.cur_c0, st.cur_c1, st.cur_n);
-            ++st.ring_n;
-            if (st.pend_n > 0) { st.op = kOpV; return true; }
-            break;                                          // no V pending: straight to the bookkeeping below
-        }
-        case kOpV: {
-            if (!mbar_test(&sc->empty[g], gph ^ 1u)) return false;
-            load_group(p, sr, tm_v, g, st.pend_bh, st.pend_c0, st.pend_c1, st.pend_n);
-            ++st.ring_n;
-            break;
-        }
-        case kOpRelease: {
-            mbar_arrive(&sc->sched_empty[ss]);
-            ++st.sched_n;
-            st.op = st.w < 0 ? (st.pend_n > 0 ? kOpFinalV : kOpDone) : kOpSlot;
-            return true;
-        }
-        case kOpFinalV: {
-            if (!mbar_test(&sc->empty[g], gph ^ 1u)) return false;
-            load_group(p, sr, tm_v, g, st.pend_bh, st.pend_c0, st.pend_c1, st.pend_n);
-            ++st.ring_n;
-            st.pend_n = 0;
-            st.op = kOpDone;
-            return true;
-        }
-        default: return false;
-    }
-    // the step's K (and the previous step's V) are on their way: this step's V becomes the pending one
-    st.pend_n = st.cur_n;
-    st.pend_bh = st.bh;
-    st.pend_c0 = st.cur_c0;
-    st.pend_c1 = st.cur_c1;
-    st.i += kStepChunks;
-    st.op = st.i < st.n ? kOpK : kOpRelease;
+// ------------------------------------------------------------------------------------------------ TMA producer (two lanes per stream)
+// Four lanes of the producer warp: per stream one fetches Q and the K blocks, the other the V blocks.  The ring
+// order of a stream is the order in which its MMA thread consumes groups, K0 K1 V0 K2 V1 K3 ...: the K blocks of
+// step t go to ring entry 2t - 1 (0 for t = 0), its V blocks to entry 2t + 2, so the two lanes never need to talk.
+// A lane cannot block (it shares its warp with the others): it polls, backing off briefly between rounds.
+__device__ __forceinline__ bool poll_wait(unsigned long long* bar, unsigned parity, IdleClock& idle, int* abort_flag, int* status, int code) {
+    while (!mbar_test(bar, parity))
+        if (!idle.tick(abort_flag, status, code, 20)) return false;
+    idle.reset();
     return true;
 }
 
-// Lane s of the producer warp serves stream s: the lanes run the same loop side by side, so that the two
-// streams' copies are issued by the same instructions most of the time.
-__device__ __forceinline__ void producer_role(const KernelParams& p, SmemCtl* ctl, const StreamRef& sr,
+__device__ __forceinline__ void producer_role(const KernelParams& p, SmemCtl* ctl, const StreamRef& sr, bool v_lane,
                                               const CUtensorMap* tm_q, const CUtensorMap* tm_k, const CUtensorMap* tm_v) {
-    ProducerState st;
+    StreamCtl* sc = sr.sc;
+    int* abort_flag = &ctl->abort_flag;
+    const CUtensorMap* tm = v_lane ? tm_v : tm_k;
+    unsigned sched_n = 0, q_n = 0, step_n = 0;      // step_n: steps of this stream seen so far
     IdleClock idle;
-    while (st.op != kOpDone) {
-        if (producer_advance(p, sr, st, tm_q, tm_k, tm_v)) idle.reset();
-        else if (!idle.tick(&ctl->abort_flag, p.status, 10, 40)) return;
+    for (;;) {
+        const unsigned ss = sched_n % kSchedSlots, sp = (sched_n / kSchedSlots) & 1u;
+        if (!poll_wait(&sc->sched_full[ss], sp, idle, abort_flag, p.status, 13)) return;
+        const WorkSlot* slot = &sc->slot[ss];
+        const int w = slot->w, flags = slot->flags, bh = slot->bh, n = slot->n_chunks;
+        if (w >= 0 && (flags & kSegLive)) {
+            if (!v_lane && (flags & kSegFirst)) {
+                const int qa = slot->qa, qb = slot->qb;
+                const unsigned qs = q_n & 1u;
+                if (!poll_wait(&sc->q_empty[qs], ((q_n >> 1) & 1u) ^ 1u, idle, abort_flag, p.status, 12)) return;
+                mbar_expect_tx(&sc->q_full[qs], qb >= 0 ? 2 * kTileBytes : kTileBytes);
+                tma_load_tile(sr.smem + kStreamSmemQ + qs * 2 * kTileBytes, tm_q, (bh * p.nb + qa) * kBlock, &sc->q_full[qs]);
+                if (qb >= 0) tma_load_tile(sr.smem + kStreamSmemQ + qs * 2 * kTileBytes + kTileBytes, tm_q, (bh * p.nb + qb) * kBlock, &sc->q_full[qs]);
+                ++q_n;
+            }
+            for (int i = 0; i < n; i += kStepChunks) {
+                const int cnt = min(kStepChunks, n - i);
+                const unsigned ring_i = v_lane ? 2u * step_n + 2u : (step_n == 0u ? 0u : 2u * step_n - 1u);
+                const unsigned g = ring_i % kRingGroups, ph = (ring_i / kRingGroups) & 1u;
+                const int c0 = slot->chunks[i].c, c1 = cnt > 1 ? slot->chunks[i + 1].c : 0;
+                if (!BB_CHECK(bh >= 0 && bh < p.BH && c0 >= 0 && c0 < p.nb && c1 >= 0 && c1 < p.nb && n <= kSegChunks, 73)) return;
+                if (!poll_wait(&sc->empty[g], ph ^ 1u, idle, abort_flag, p.status, 10)) return;
+                mbar_expect_tx(&sc->full[g], cnt * kTileBytes);
+                tma_load_tile(sr.smem + kStreamSmemRing + g * kGroupBytes, tm, (bh * p.nb + c0) * kBlock, &sc->full[g]);
+                if (cnt > 1) tma_load_tile(sr.smem + kStreamSmemRing + g * kGroupBytes + kTileBytes, tm, (bh * p.nb + c1) * kBlock, &sc->full[g]);
+                ++step_n;
+            }
+        }
+        mbar_arrive(&sc->sched_empty[ss]);
+        ++sched_n;
+        if (w < 0) return;
     }
 }
 
@@ -633,11 +595,13 @@ __device__ __forceinline__ void producer_role(const KernelParams& p, SmemCtl* ct
 __device__ __forceinline__ void mma_role(const KernelParams& p, SmemCtl* ctl, const StreamRef& sr) {
     StreamCtl* sc = sr.sc;
     int* abort_flag = &ctl->abort_flag;
-    unsigned ring_n = 0, q_n = 0, sched_n = 0, grp_n = 0, pv_n = 0, tile_n = 0;   // grp_n: steps whose Q K^T was issued; tile_n: tiles handed to the epilogue
+    unsigned q_n = 0, sched_n = 0, grp_n = 0, pv_n = 0, tile_n = 0;   // grp_n: steps whose Q K^T was issued; tile_n: tiles handed to the epilogue
     bool ok = true;
     int fail = 0;                               // code of the wait that was abandoned, if any
-    auto qk = [&](int cnt, unsigned qs) -> bool {   // S[:, 0 .. 64 cnt) = Q K^T with the K blocks of the next ring group
-        const unsigned g = ring_n % kRingGroups, ph = (ring_n / kRingGroups) & 1u;
+    // ring entries (see the producer): the K blocks of step t sit in entry 2t - 1 (0 for t = 0), its V blocks in 2t + 2
+    auto qk = [&](int cnt, unsigned qs) -> bool {   // S[:, 0 .. 64 cnt) = Q K^T with the K blocks of step grp_n
+        const unsigned ring_i = grp_n == 0u ? 0u : 2u * grp_n - 1u;
+        const unsigned g = ring_i % kRingGroups, ph = (ring_i / kRingGroups) & 1u;
         if (!mbar_wait(&sc->full[g], ph, abort_flag)) { fail = 20; return false; }
         tc_fence_after();
         // the blocks of a group are adjacent: their 64 cnt rows form one K-major operand
@@ -648,7 +612,6 @@ __device__ __forceinline__ void mma_role(const KernelParams& p, SmemCtl* ctl, co
         for (int kk = 0; kk < 4; ++kk)          // 16 head dims (32 bytes inside the swizzled row) per MMA
             mma_ss(sr.tmem + kColS, q_desc + (unsigned long long)(kk * 2), k_desc + (unsigned long long)(kk * 2), idesc, kk > 0);
         tc_commit(&sc->empty[g]);
-        ++ring_n;
         return true;
     };
     bool pend_fresh = false;                    // the pending P V is the first of its tile: it overwrites O
@@ -660,7 +623,8 @@ __device__ __forceinline__ void mma_role(const KernelParams& p, SmemCtl* ctl, co
         if (!mbar_wait(&sc->p_full, pv_n & 1u, abort_flag)) { fail = 22; return false; }
         // the epilogue must have taken the previous tile's accumulator before this tile's first P V overwrites it
         if (pend_fresh && tile_n > 0 && !mbar_wait(&sc->o_free, (tile_n - 1) & 1u, abort_flag)) { fail = 27; return false; }
-        const unsigned g = ring_n % kRingGroups, ph = (ring_n / kRingGroups) & 1u;
+        const unsigned ring_i = 2u * pv_n + 2u;
+        const unsigned g = ring_i % kRingGroups, ph = (ring_i / kRingGroups) & 1u;
         if (!mbar_wait(&sc->full[g], ph, abort_flag)) { fail = 21; return false; }
         tc_fence_after();
         const unsigned long long v_desc = smem_desc_sw128(smem_u32(sr.smem + kStreamSmemRing + g * kGroupBytes));
@@ -679,7 +643,6 @@ __device__ __forceinline__ void mma_role(const KernelParams& p, SmemCtl* ctl, co
             tc_commit(&sc->o_done);
             ++tile_n;
         }
-        ++ring_n;
         ++pv_n;
         pend_n = 0;
         pend_fresh = false;
@@ -945,7 +908,8 @@ __device__ __forceinline__ void epilogue_role(const KernelParams& p, SmemCtl* ct
             const bool partial = part_slot >= 0;
             unsigned char* dst = partial ? reinterpret_cast<unsigned char*>(p.partials + (size_t)part_slot * kPartialFloats + row * 64)
                                          : reinterpret_cast<unsigned char*>(p.out + (((size_t)bh * p.nb + (my_q >= 0 ? my_q : 0)) * kBlock + r64) * kBlock);
-            const bool write = partial || my_q >= 0;        // warp-uniform
+            bool write = partial || my_q >= 0;              // warp-uniform
+            if (!BB_CHECK(bh >= 0 && bh < p.BH && my_q < p.nb && part_slot < p.BH * max(p.split_tiles_per_head, 1) * p.max_parts, 74)) write = false;
 #pragma unroll 1
             for (int c = 0; c < 2; ++c) {
                 float o[32];
@@ -1002,7 +966,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             mbar_init(&sc->pv_done, 1);
             mbar_init(&sc->o_done, 1);
             mbar_init(&sc->o_free, kSoftmaxThreads);    // the 128 epilogue threads
-            for (int i = 0; i < kSchedSlots; ++i) { mbar_init(&sc->sched_full[i], 1); mbar_init(&sc->sched_empty[i], 2 + kSoftmaxThreads); }
+            for (int i = 0; i < kSchedSlots; ++i) { mbar_init(&sc->sched_full[i], 1); mbar_init(&sc->sched_empty[i], 3 + kSoftmaxThreads); }    // two producer lanes, the MMA thread, the softmax threads
         }
         ctl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -1028,7 +992,7 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
     } else {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsLight));
         if (warp == kWarpScheduler) scheduler_role(p, ctl, lane);
-        else if (warp == kWarpProducer) { if (lane < kStreams) producer_role(p, ctl, lane == 0 ? s0 : s1, &tm_q, &tm_k, &tm_v); }
+        else if (warp == kWarpProducer) { if (lane < 2 * kStreams) producer_role(p, ctl, (lane & 1) ? s1 : s0, lane >= kStreams, &tm_q, &tm_k, &tm_v); }
         else if (lane == 0) mma_role(p, ctl, warp == kWarpMma ? s0 : s1);
     }
 

@@ -250,6 +250,7 @@ const char* bigbird_strerror(int code) {
         case BIGBIRD_ETIMEOUT: return "bounded device wait expired";
         case BIGBIRD_ENOMEM: return "out of memory";
         case BIGBIRD_ELIMIT: return "problem exceeds the fixed scratch of the no-allocation entry point";
+        case BIGBIRD_EINTERNAL: return "index check failed inside a kernel (checked build)";
         default: return "unknown error";
     }
 }
