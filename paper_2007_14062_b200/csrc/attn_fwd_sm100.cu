@@ -203,6 +203,9 @@ __device__ __forceinline__ bool mbar_test(unsigned long long* bar, unsigned pari
 // thread of the CTA has given up; the caller leaves its loop and calls give_up with the code of the wait.
 constexpr unsigned kWaitTries = 1500000;
 __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned parity, int* abort_flag) {
+    // a phase that is already complete is seen by the plain test in a dozen cycles; try_wait, which may put the
+    // thread to sleep, takes a few hundred even then (measured on the MMA thread's time line)
+    if (mbar_test(bar, parity)) return true;
 #pragma unroll 1
     for (unsigned it = 0; it < kWaitTries; ++it) {
         if (mbar_try(bar, parity)) return true;
@@ -281,6 +284,21 @@ __device__ __forceinline__ void mma_ts(unsigned d_tmem, unsigned a_tmem, unsigne
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
         ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+// The same, issued only if enable != 0 (a predicated instruction instead of a branch around it: a lone thread pays
+// for every branch it executes with a stall until the target is known).
+__device__ __forceinline__ void mma_ts_if(unsigned d_tmem, unsigned a_tmem, unsigned long long b_desc, unsigned idesc, unsigned accumulate, unsigned enable) {
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 p, %4, 0;\n\tsetp.ne.b32 q, %5, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(enable) : "memory");
+}
+__device__ __forceinline__ void tc_commit_if(unsigned long long* bar, unsigned enable) {
+    asm volatile(
+        "{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %1, 0;\n\t"
+        "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+        ::"r"(smem_u32(bar)), "r"(enable) : "memory");
 }
 
 // Shared-memory matrix descriptor, 128-byte swizzle, 8-row groups 1024 bytes apart (a dense 64-wide bf16 tile).
@@ -381,6 +399,28 @@ __device__ __forceinline__ void fadd2(float& r0, float& r1, float x0, float x1) 
 __device__ __forceinline__ void fmul2(float& r0, float& r1, float a) {
     asm("{ .reg .b64 ra, rb, rd; mov.b64 ra, {%0, %1}; mov.b64 rb, {%2, %2}; mul.f32x2 rd, ra, rb; mov.b64 {%0, %1}, rd; }"
         : "+f"(r0), "+f"(r1) : "f"(a));
+}
+
+// Order-preserving twins of the wrappers above (volatile: the compiler keeps them in source order), for the one loop
+// whose instruction order is laid out by hand.
+__device__ __forceinline__ float ex2_o(float x) {
+    float y;
+    asm volatile("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ unsigned pack_bf16_o(float lo, float hi) {
+    unsigned d;
+    asm volatile("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+__device__ __forceinline__ void ffma2_o(float& r0, float& r1, float x0, float x1, float a, float b) {
+    asm volatile("{ .reg .b64 ra, rb, rc, rd; mov.b64 ra, {%2, %3}; mov.b64 rb, {%4, %4}; mov.b64 rc, {%5, %5}; "
+                 "fma.rn.f32x2 rd, ra, rb, rc; mov.b64 {%0, %1}, rd; }"
+                 : "=f"(r0), "=f"(r1) : "f"(x0), "f"(x1), "f"(a), "f"(b));
+}
+__device__ __forceinline__ void fadd2_o(float& r0, float& r1, float x0, float x1) {
+    asm volatile("{ .reg .b64 ra, rb, rd; mov.b64 ra, {%0, %1}; mov.b64 rb, {%2, %3}; add.f32x2 rd, ra, rb; mov.b64 {%0, %1}, rd; }"
+                 : "+f"(r0), "+f"(r1) : "f"(x0), "f"(x1));
 }
 
 // ------------------------------------------------------------------------------------------------ helpers
@@ -592,116 +632,100 @@ __device__ __forceinline__ void producer_role(const KernelParams& p, SmemCtl* ct
 }
 
 // ------------------------------------------------------------------------------------------------ MMA issuer (one thread per stream)
+// One thread per stream walks the posted slots; a round issues S = Q K^T of a step and, behind it, O += P V of the
+// step before (whose probabilities the softmax threads were writing meanwhile).  The thread is alone in its warp, so
+// nothing hides its latencies: every branch stalls it until the target is known and every barrier test is a round
+// trip to shared memory.  Hence the shape of the loop: the two barriers a product needs are tested back to back and
+// one branch takes the combined result; a second key block and the end of a tile are predicated instructions.
+// Ring entries (see the producer): the K blocks of step t sit in entry 2t - 1 (0 for t = 0), its V blocks in 2t + 2.
 __device__ __forceinline__ void mma_role(const KernelParams& p, SmemCtl* ctl, const StreamRef& sr) {
     StreamCtl* sc = sr.sc;
     int* abort_flag = &ctl->abort_flag;
     unsigned q_n = 0, sched_n = 0, grp_n = 0, pv_n = 0, tile_n = 0;   // grp_n: steps whose Q K^T was issued; tile_n: tiles handed to the epilogue
-    bool ok = true;
     int fail = 0;                               // code of the wait that was abandoned, if any
-    // ring entries (see the producer): the K blocks of step t sit in entry 2t - 1 (0 for t = 0), its V blocks in 2t + 2
-    auto qk = [&](int cnt, unsigned qs) -> bool {   // S[:, 0 .. 64 cnt) = Q K^T with the K blocks of step grp_n
-        const unsigned ring_i = grp_n == 0u ? 0u : 2u * grp_n - 1u;
-        const unsigned g = ring_i % kRingGroups, ph = (ring_i / kRingGroups) & 1u;
-        if (!mbar_wait(&sc->full[g], ph, abort_flag)) { fail = 20; return false; }
-        tc_fence_after();
-        // the blocks of a group are adjacent: their 64 cnt rows form one K-major operand
-        const unsigned long long q_desc = smem_desc_sw128(smem_u32(sr.smem + kStreamSmemQ + qs * 2 * kTileBytes));
-        const unsigned long long k_desc = smem_desc_sw128(smem_u32(sr.smem + kStreamSmemRing + g * kGroupBytes));
-        const unsigned idesc = kIdescQK64 + ((unsigned)(cnt - 1) << 20);           // N = 64 cnt
-#pragma unroll
-        for (int kk = 0; kk < 4; ++kk)          // 16 head dims (32 bytes inside the swizzled row) per MMA
-            mma_ss(sr.tmem + kColS, q_desc + (unsigned long long)(kk * 2), k_desc + (unsigned long long)(kk * 2), idesc, kk > 0);
-        tc_commit(&sc->empty[g]);
-        return true;
-    };
-    bool pend_fresh = false;                    // the pending P V is the first of its tile: it overwrites O
+    unsigned pend_cnt = 0;                      // key blocks of the step whose P V is still to be issued (0: none)
+    bool pend_fresh = false;                    // ... it is the first of its tile: it overwrites O
     bool pend_last = false;                     // ... the last of its tile: the accumulator is complete after it
-    bool tile_fresh = false, q_unseen = false;
-    int pend_n = 0, tile_steps = 0;
-    auto pending_pv = [&]() -> bool {           // O (+)= sum_j P_j V_j with the V blocks of the next ring group
-        if (pend_n == 0) return true;
-        if (!mbar_wait(&sc->p_full, pv_n & 1u, abort_flag)) { fail = 22; return false; }
-        // the epilogue must have taken the previous tile's accumulator before this tile's first P V overwrites it
-        if (pend_fresh && tile_n > 0 && !mbar_wait(&sc->o_free, (tile_n - 1) & 1u, abort_flag)) { fail = 27; return false; }
-        const unsigned ring_i = 2u * pv_n + 2u;
-        const unsigned g = ring_i % kRingGroups, ph = (ring_i / kRingGroups) & 1u;
-        if (!mbar_wait(&sc->full[g], ph, abort_flag)) { fail = 21; return false; }
-        tc_fence_after();
-        const unsigned long long v_desc = smem_desc_sw128(smem_u32(sr.smem + kStreamSmemRing + g * kGroupBytes));
-#pragma unroll 1
-        for (int j = 0; j < pend_n; ++j) {
-            {
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk)  // 16 keys per MMA: 8 packed columns of P_j, two 8-row groups of V_j
-                    mma_ts(sr.tmem + kColO, sr.tmem + kColP + 32 * j + kk * 8, v_desc + (unsigned long long)((j * kTileBytes + kk * 2048) >> 4), kIdescPV,
-                           (j > 0 || kk > 0 || !pend_fresh) ? 1u : 0u);
-            }
-        }
-        tc_commit(&sc->empty[g]);
-        tc_commit(&sc->pv_done);
-        if (pend_last) {
-            tc_commit(&sc->o_done);
-            ++tile_n;
-        }
-        ++pv_n;
-        pend_n = 0;
-        pend_fresh = false;
-        pend_last = false;
+    bool tile_steps = false;                    // the current tile has had a step
+    const unsigned q_base = smem_u32(sr.smem + kStreamSmemQ), ring_base = smem_u32(sr.smem + kStreamSmemRing);
+    // both barriers at once; the blocking waits only if one of them is not there yet
+    auto wait2 = [&](unsigned long long* b1, unsigned par1, bool need1, int code1, unsigned long long* b2, unsigned par2, int code2) -> bool {
+        const bool t1 = mbar_test(b1, par1), t2 = mbar_test(b2, par2);
+        if (__builtin_expect((t1 || !need1) && t2, 1)) return true;
+        if (need1 && !mbar_wait(b1, par1, abort_flag)) { fail = code1; return false; }
+        if (!mbar_wait(b2, par2, abort_flag)) { fail = code2; return false; }
         return true;
     };
-    while (ok) {
+    for (;;) {
         const unsigned ss = sched_n % kSchedSlots, sp = (sched_n / kSchedSlots) & 1u;
         if (!mbar_wait(&sc->sched_full[ss], sp, abort_flag)) { fail = 23; break; }
         const WorkSlot* slot = &sc->slot[ss];
         const int w = slot->w, flags = slot->flags, n = slot->n_chunks;
-        if (w >= 0 && (flags & kSegLive) && (flags & kSegFirst)) {
-            ++q_n;                              // this tile's Q sits in buffer (q_n - 1) & 1
-            q_unseen = true;
-            tile_fresh = true;
-            tile_steps = 0;
-        }
         const bool work = w >= 0 && (flags & kSegLive);
-        const unsigned qs = (q_n - 1) & 1u, qph = ((q_n - 1) >> 1) & 1u;
-        // one round per step of the slot: this step's Q K^T, then the previous step's P V behind it; the slot that
-        // says "no more work" gets one round without a Q K^T, which issues the very last P V
+        const bool first = work && (flags & kSegFirst), last = work && (flags & kSegLast);
+        if (first) {
+            tile_steps = false;
+            ++q_n;                              // this tile's Q sits in buffer (q_n - 1) & 1
+            if (!mbar_wait(&sc->q_full[(q_n - 1) & 1u], ((q_n - 1) >> 1) & 1u, abort_flag)) { fail = 24; break; }
+        }
+        const unsigned qs = (q_n - 1) & 1u;
+        const unsigned long long q_desc = smem_desc_sw128(q_base + qs * 2 * kTileBytes);
+        // one round per step of the slot; the slot that says "no more work" gets one round without a Q K^T, which
+        // issues the very last P V
         const int n_rounds = work ? (n + kStepChunks - 1) / kStepChunks : (w < 0 ? 1 : 0);
-        for (int r = 0; r < n_rounds && ok; ++r) {
-            int cnt = 0;
-            if (work) {
-                // the softmax threads must have pulled the previous scores out of tensor memory
-                if (grp_n > 0) {
-                    ok = mbar_wait(&sc->s_free, (grp_n - 1) & 1u, abort_flag);
-                    if (!ok) { fail = 25; break; }
-                }
-                if (q_unseen) {
-                    ok = mbar_wait(&sc->q_full[qs], qph, abort_flag);
-                    if (!ok) { fail = 24; break; }
-                    q_unseen = false;
-                }
+        bool tile_fresh = first;
+#pragma unroll 1
+        for (int r = 0; r < n_rounds; ++r) {
+            const unsigned cnt = work ? (unsigned)min(kStepChunks, n - r * kStepChunks) : 0u;
+            if (cnt) {
+                // S[:, 0 .. 64 cnt) = Q K^T: the softmax threads must have pulled the previous scores out of tensor
+                // memory, and the K blocks must have landed
+                const unsigned ring_i = grp_n == 0u ? 0u : 2u * grp_n - 1u;
+                const unsigned g = ring_i % kRingGroups, ph = (ring_i / kRingGroups) & 1u;
+                // the blocks of a group are adjacent: their 64 cnt rows form one K-major operand
+                const unsigned long long k_desc = smem_desc_sw128(ring_base + g * kGroupBytes);
+                const unsigned idesc = kIdescQK64 + ((cnt - 1u) << 20);                    // N = 64 cnt
+                if (!wait2(&sc->s_free, (grp_n - 1u) & 1u, grp_n > 0u, 25, &sc->full[g], ph, 20)) break;
                 tc_fence_after();
-                cnt = min(kStepChunks, n - r * kStepChunks);
-                ok = qk(cnt, qs);
-                if (!ok) break;
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)  // 16 head dims (32 bytes inside the swizzled row) per MMA
+                    mma_ss(sr.tmem + kColS, q_desc + (unsigned long long)(kk * 2), k_desc + (unsigned long long)(kk * 2), idesc, kk > 0);
                 tc_commit(&sc->s_full);
+                tc_commit(&sc->empty[g]);
                 ++grp_n;
             }
-            ok = pending_pv();
-            if (work) {
-                pend_n = cnt;
-                pend_fresh = tile_fresh;
-                tile_fresh = false;
-                ++tile_steps;
+            if (pend_cnt) {
+                // O (+)= sum_j P_j V_j with the V blocks of the pending step
+                const unsigned ring_i = 2u * pv_n + 2u;
+                const unsigned g = ring_i % kRingGroups, ph = (ring_i / kRingGroups) & 1u;
+                const unsigned long long v_desc = smem_desc_sw128(ring_base + g * kGroupBytes);
+                const unsigned acc0 = pend_fresh ? 0u : 1u, two = pend_cnt > 1u ? 1u : 0u;
+                // the epilogue must have taken the previous tile's accumulator before this tile's first P V overwrites it
+                if (pend_fresh && tile_n > 0 && !mbar_wait(&sc->o_free, (tile_n - 1) & 1u, abort_flag)) { fail = 27; break; }
+                if (!wait2(&sc->p_full, pv_n & 1u, true, 22, &sc->full[g], ph, 21)) break;
+                tc_fence_after();
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)  // 16 keys per MMA: 8 packed columns of P_j, two 8-row groups of V_j
+                    mma_ts(sr.tmem + kColO, sr.tmem + kColP + kk * 8, v_desc + (unsigned long long)((kk * 2048) >> 4), kIdescPV, kk > 0 ? 1u : acc0);
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)
+                    mma_ts_if(sr.tmem + kColO, sr.tmem + kColP + 32 + kk * 8, v_desc + (unsigned long long)((kTileBytes + kk * 2048) >> 4), kIdescPV, 1u, two);
+                tc_commit(&sc->pv_done);
+                tc_commit_if(&sc->o_done, pend_last ? 1u : 0u);
+                tc_commit(&sc->empty[g]);
+                tile_n += pend_last ? 1u : 0u;
+                ++pv_n;
             }
+            pend_cnt = cnt;
+            pend_fresh = tile_fresh;
+            pend_last = false;
+            tile_fresh = tile_fresh && cnt == 0u;
+            tile_steps = tile_steps || cnt != 0u;
         }
-        if (!ok) break;
-        if (work && (flags & kSegLast)) {
-            if (q_unseen) {                     // a tile without a live key block: its Q still has to land
-                ok = mbar_wait(&sc->q_full[qs], qph, abort_flag);
-                if (!ok) { fail = 26; break; }
-                q_unseen = false;
-            }
-            tc_commit(&sc->q_empty[qs]);       // every Q K^T of the tile has been issued
-            if (tile_steps > 0) pend_last = true;           // the tile's last P V is the pending one
+        if (fail) break;
+        if (last) {
+            tc_commit(&sc->q_empty[qs]);        // every Q K^T of the tile has been issued
+            pend_last = tile_steps;             // the tile's last P V is the pending one (the tile's last segment may be empty)
         }
         mbar_arrive(&sc->sched_empty[ss]);
         ++sched_n;
@@ -727,15 +751,30 @@ __device__ __forceinline__ void softmax_role(const KernelParams& p, SmemCtl* ctl
     bool o_dirty = false;                           // has any P V been issued for this tile yet
     // exponentials of the 64 scores of one key block, packed in place: afterwards s[0..31] hold the bit
     // patterns of the 32 words of bf16 probability pairs
+    // A warp issues in order, and an exponential holds the special-function unit for eight cycles: unless other work
+    // sits between two of them in the instruction stream, the warp just waits.  So the order is laid out by hand,
+    // as a software pipeline over the 32 pairs: exponential of pair j (low half), scale-and-shift of pair j + 2,
+    // exponential of pair j (high half), sum and pack of pair j - 1.
     auto exp_pack = [&](float* s, float neg_m, float& sum0, float& sum1) {
+        float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f;
+        float x[3][2], pr[2][2];
+        ffma2_o(x[0][0], x[0][1], s[0], s[1], sl2, neg_m);
+        ffma2_o(x[1][0], x[1][1], s[2], s[3], sl2, neg_m);
 #pragma unroll
-        for (int t = 0; t < 64; t += 2) {
-            float t0, t1;
-            ffma2(t0, t1, s[t], s[t + 1], sl2, neg_m);
-            const float p0 = ex2(t0), p1 = ex2(t1);
-            fadd2(sum0, sum1, p0, p1);
-            s[t >> 1] = __uint_as_float(pack_bf16(p0, p1));
+        for (int j = 0; j < 32; ++j) {
+            pr[j & 1][0] = ex2_o(x[j % 3][0]);
+            if (j + 2 < 32) ffma2_o(x[(j + 2) % 3][0], x[(j + 2) % 3][1], s[2 * j + 4], s[2 * j + 5], sl2, neg_m);
+            pr[j & 1][1] = ex2_o(x[j % 3][1]);
+            if (j >= 1) {
+                if (j & 1) fadd2_o(b0, b1, pr[(j - 1) & 1][0], pr[(j - 1) & 1][1]);
+                else fadd2_o(a0, a1, pr[(j - 1) & 1][0], pr[(j - 1) & 1][1]);
+                s[j - 1] = __uint_as_float(pack_bf16_o(pr[(j - 1) & 1][0], pr[(j - 1) & 1][1]));
+            }
         }
+        fadd2_o(b0, b1, pr[1][0], pr[1][1]);
+        s[31] = __uint_as_float(pack_bf16_o(pr[1][0], pr[1][1]));
+        fadd2_o(a0, a1, b0, b1);
+        fadd2_o(sum0, sum1, a0, a1);
     };
     while (ok) {
         const unsigned ss = sched_n % kSchedSlots, sp = (sched_n / kSchedSlots) & 1u;
