@@ -57,15 +57,17 @@ constexpr int kStreams = 2;                // tile streams per CTA
 constexpr int kThreads = 512;
 constexpr int kWarpEpilogue = 8, kWarpProducer = 12, kWarpMma = 13, kWarpScheduler = 15;
 constexpr int kSoftmaxThreads = 128;
-// 512 threads x 128 registers fill the register file; no role needs more (the softmax threads hold one key block's
-// scores at a time), so the register split between roles stays even and nothing spills: a spill here costs a trip
-// to L2, since nearly all of the SM's L1 is configured as shared memory.
+// 512 threads start with 128 registers each; the roles then trade.  A sub-partition's registers are shared out
+// among its own four warps only (setmaxnreg can hand out no more than those warps gave back): two softmax warps x 200
+// (a step's 128 scores plus the loop's temporaries) + an epilogue warp x 56 + a light warp x 56 = 4 x 128 exactly.
+// Nothing may spill: a spill here costs a trip to L2, since nearly all of the SM's L1 is configured as shared memory.
 #ifndef BB_REGS_SOFTMAX
-#define BB_REGS_SOFTMAX 184
-#define BB_REGS_EPILOGUE 80
-#define BB_REGS_LIGHT 64
+#define BB_REGS_SOFTMAX 200
+#define BB_REGS_EPILOGUE 56
+#define BB_REGS_LIGHT 56
 #endif
 constexpr int kRegsSoftmax = BB_REGS_SOFTMAX, kRegsEpilogue = BB_REGS_EPILOGUE, kRegsLight = BB_REGS_LIGHT;
+static_assert(2 * kRegsSoftmax + kRegsEpilogue + kRegsLight <= 4 * 128 && kThreads == 512, "register trade between the four warps of a sub-partition");
 constexpr int kTmemCols = 512;
 constexpr int kStreamCols = kTmemCols / kStreams;
 constexpr int kColS = 0;                   // scores: kStepChunks x 64 fp32 columns
@@ -173,18 +175,6 @@ __device__ __forceinline__ unsigned long long global_ns() {
     return t;
 }
 
-// One try with a time hint.  On this part a failing try with a hint keeps the thread suspended for about 4 us
-// whatever the hint says (measured), and wakes early when the phase completes: a role that watches two barriers uses
-// it to sleep on one of them between rounds instead of spinning.
-__device__ __forceinline__ bool mbar_try_for(unsigned long long* bar, unsigned parity, unsigned ns) {
-    unsigned ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(ns) : "memory");
-    return ok != 0;
-}
 // Non-blocking test of a phase (for the roles that poll several barriers).
 __device__ __forceinline__ bool mbar_test(unsigned long long* bar, unsigned parity) {
     unsigned ok;
@@ -399,28 +389,6 @@ __device__ __forceinline__ void fadd2(float& r0, float& r1, float x0, float x1) 
 __device__ __forceinline__ void fmul2(float& r0, float& r1, float a) {
     asm("{ .reg .b64 ra, rb, rd; mov.b64 ra, {%0, %1}; mov.b64 rb, {%2, %2}; mul.f32x2 rd, ra, rb; mov.b64 {%0, %1}, rd; }"
         : "+f"(r0), "+f"(r1) : "f"(a));
-}
-
-// Order-preserving twins of the wrappers above (volatile: the compiler keeps them in source order), for the one loop
-// whose instruction order is laid out by hand.
-__device__ __forceinline__ float ex2_o(float x) {
-    float y;
-    asm volatile("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-__device__ __forceinline__ unsigned pack_bf16_o(float lo, float hi) {
-    unsigned d;
-    asm volatile("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
-    return d;
-}
-__device__ __forceinline__ void ffma2_o(float& r0, float& r1, float x0, float x1, float a, float b) {
-    asm volatile("{ .reg .b64 ra, rb, rc, rd; mov.b64 ra, {%2, %3}; mov.b64 rb, {%4, %4}; mov.b64 rc, {%5, %5}; "
-                 "fma.rn.f32x2 rd, ra, rb, rc; mov.b64 {%0, %1}, rd; }"
-                 : "=f"(r0), "=f"(r1) : "f"(x0), "f"(x1), "f"(a), "f"(b));
-}
-__device__ __forceinline__ void fadd2_o(float& r0, float& r1, float x0, float x1) {
-    asm volatile("{ .reg .b64 ra, rb, rd; mov.b64 ra, {%0, %1}; mov.b64 rb, {%2, %3}; add.f32x2 rd, ra, rb; mov.b64 {%0, %1}, rd; }"
-                 : "+f"(r0), "+f"(r1) : "f"(x0), "f"(x1));
 }
 
 // ------------------------------------------------------------------------------------------------ helpers
@@ -750,31 +718,21 @@ __device__ __forceinline__ void softmax_role(const KernelParams& p, SmemCtl* ctl
     float m_ref = -INFINITY, l_sum = 0.f;
     bool o_dirty = false;                           // has any P V been issued for this tile yet
     // exponentials of the 64 scores of one key block, packed in place: afterwards s[0..31] hold the bit
-    // patterns of the 32 words of bf16 probability pairs
-    // A warp issues in order, and an exponential holds the special-function unit for eight cycles: unless other work
-    // sits between two of them in the instruction stream, the warp just waits.  So the order is laid out by hand,
-    // as a software pipeline over the 32 pairs: exponential of pair j (low half), scale-and-shift of pair j + 2,
-    // exponential of pair j (high half), sum and pack of pair j - 1.
+    // patterns of the 32 words of bf16 probability pairs (four partial sums, so that the adds do not form one chain)
     auto exp_pack = [&](float* s, float neg_m, float& sum0, float& sum1) {
         float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f;
-        float x[3][2], pr[2][2];
-        ffma2_o(x[0][0], x[0][1], s[0], s[1], sl2, neg_m);
-        ffma2_o(x[1][0], x[1][1], s[2], s[3], sl2, neg_m);
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
-            pr[j & 1][0] = ex2_o(x[j % 3][0]);
-            if (j + 2 < 32) ffma2_o(x[(j + 2) % 3][0], x[(j + 2) % 3][1], s[2 * j + 4], s[2 * j + 5], sl2, neg_m);
-            pr[j & 1][1] = ex2_o(x[j % 3][1]);
-            if (j >= 1) {
-                if (j & 1) fadd2_o(b0, b1, pr[(j - 1) & 1][0], pr[(j - 1) & 1][1]);
-                else fadd2_o(a0, a1, pr[(j - 1) & 1][0], pr[(j - 1) & 1][1]);
-                s[j - 1] = __uint_as_float(pack_bf16_o(pr[(j - 1) & 1][0], pr[(j - 1) & 1][1]));
-            }
+            float x0, x1, p0, p1;
+            ffma2(x0, x1, s[2 * j], s[2 * j + 1], sl2, neg_m);
+            p0 = ex2(x0);
+            p1 = ex2(x1);
+            if (j & 1) fadd2(b0, b1, p0, p1);
+            else fadd2(a0, a1, p0, p1);
+            s[j] = __uint_as_float(pack_bf16(p0, p1));
         }
-        fadd2_o(b0, b1, pr[1][0], pr[1][1]);
-        s[31] = __uint_as_float(pack_bf16_o(pr[1][0], pr[1][1]));
-        fadd2_o(a0, a1, b0, b1);
-        fadd2_o(sum0, sum1, a0, a1);
+        fadd2(a0, a1, b0, b1);
+        fadd2(sum0, sum1, a0, a1);
     };
     while (ok) {
         const unsigned ss = sched_n % kSchedSlots, sp = (sched_n / kSchedSlots) & 1u;
@@ -976,10 +934,9 @@ __device__ __forceinline__ void epilogue_role(const KernelParams& p, SmemCtl* ct
         }
         if (progress) idle.reset();
         else {
-            // suspended on stream 0's next message for a short while; stream 1's is looked at again afterwards
-            const unsigned st0 = state0;
-            if (!(st0 >> 31)) mbar_try_for(&ctl->st[0].epi_full[st0 & 1u], (st0 >> 1) & 1u, 300);
-            else __nanosleep(300);
+            // (a short sleep, not a suspended wait on one stream's barrier: that would not see the other stream's
+            // message for up to 4 us, and the stream's next tile cannot overwrite the accumulator before it is taken)
+            __nanosleep(400);
             if (!__all_sync(0xffffffffu, idle.tick(abort_flag, p.status, 41, 0))) return;
         }
     }
@@ -1000,8 +957,8 @@ attn_fwd_sm100_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             for (int i = 0; i < kRingGroups; ++i) { mbar_init(&sc->full[i], 1); mbar_init(&sc->empty[i], 1); }
             for (int i = 0; i < 2; ++i) { mbar_init(&sc->q_full[i], 1); mbar_init(&sc->q_empty[i], 1); mbar_init(&sc->epi_full[i], kSoftmaxThreads); }
             mbar_init(&sc->s_full, 1);
-            mbar_init(&sc->s_free, kSoftmaxThreads);    // every softmax thread arrives itself: cheaper than
-            mbar_init(&sc->p_full, kSoftmaxThreads);    // converging the warp and electing a lane
+            mbar_init(&sc->s_free, kSoftmaxThreads);    // every softmax thread arrives itself: converging the warp and
+            mbar_init(&sc->p_full, kSoftmaxThreads);    // electing a lane was measured 10% slower on the whole kernel
             mbar_init(&sc->pv_done, 1);
             mbar_init(&sc->o_done, 1);
             mbar_init(&sc->o_free, kSoftmaxThreads);    // the 128 epilogue threads
