@@ -36,7 +36,7 @@ NOMINAL_BF16_TFLOPS = 2250.0
 FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "hbm_gbs": 6650.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one attn_fwd_sm100_kernel launch on this workload, from the
 # ncu capture summarised in profiles/ (None until a capture exists for the current kernel).
-NCU_DRAM_BYTES_PER_LAUNCH = {"c2_base_itc_bf16": 251.4e6}
+NCU_DRAM_BYTES_PER_LAUNCH = {"c2_base_itc_bf16": 241.1e6}
 
 
 def measured_peaks():
@@ -49,9 +49,22 @@ def measured_peaks():
     return dict(FALLBACK_PEAKS, bf16_tflops_sustained=1400.0, source="fallback")
 
 
-def counted_pairs(layout, wl) -> int:
-    """Attended (query block, key block) pairs per batch element, summed over heads."""
+def counted_pairs(layout) -> int:
+    """Attended (query block, key block) pairs per batch element, summed over heads (the nominal count: every pair
+    of the layout, App. D's cost formula O(n (g + w + r) b d))."""
     return int(layout.nnz)
+
+
+def effective_pairs(layout, wl, kpm) -> int:
+    """Pairs of the whole batch that survive the key-padding mask: the query block has at least one valid row and
+    the key block at least one valid key.  Equal to B x nominal when nothing is padded."""
+    if kpm is None:
+        return wl.B * counted_pairs(layout)
+    nb = wl.N // wl.b
+    valid = kpm.numpy().reshape(wl.B, nb, wl.b).any(axis=2)                 # [B, nb]
+    row_ptr, col_idx = layout.export()
+    rows = np.repeat(np.arange(wl.H * nb), np.diff(row_ptr)) % nb          # query block of every pair
+    return int((valid[:, rows] & valid[:, col_idx]).sum())
 
 
 class ClockSampler:
@@ -120,6 +133,14 @@ def whole_job_value(per_replica_units, world, slowest_ms):
     return world * per_replica_units / (slowest_ms * 1e-3)
 
 
+def workload_config(wl, pairs_per_batch):
+    """The keys both arms report for the workload (same names, same values)."""
+    return {"workload": wl.name, "B": wl.B, "H": wl.H, "N": wl.N, "D": wl.D, "block": wl.b, "window_blocks": wl.w,
+            "global_blocks": wl.g, "random_blocks": wl.r, "mode": "ETC" if wl.mode else "ITC",
+            "attended_block_pairs_per_step": wl.B * pairs_per_batch,
+            "counted_gflop_per_step": wl.B * pairs_per_batch * 4.0 * wl.b * wl.b * wl.D / 1e9}
+
+
 def oracle_slices(wl, q, k, v, kpm, slices):
     from oracle import bigbird_oracle as O
     gr = O.Graph(wl.N, wl.b, wl.w, wl.g, wl.r, wl.seed, wl.H, wl.mode)
@@ -181,7 +202,7 @@ def run_reference(args, wl):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "N": wl.N, "D": wl.D, "block": wl.b, "sample": sample},
+        "config": dict(workload_config(wl, int(row_ptr[-1])), sample=sample),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -191,8 +212,8 @@ def run_reference(args, wl):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=4000)
-    ap.add_argument("--warmup", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=None, help="timed steps (default 1000; 12 for --impl reference)")
+    ap.add_argument("--warmup", type=int, default=None, help="untimed steps before them (default 50; 3 for --impl reference)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2_base_itc_bf16", choices=synth.ORDER)
     ap.add_argument("--e2e-steps", type=int, default=20)
@@ -201,12 +222,12 @@ def main():
     wl = synth.WORKLOADS[args.workload]
 
     if args.impl == "reference":
-        if args.steps == 4000:
-            args.steps, args.warmup = 12, 3
+        args.steps = 12 if args.steps is None else args.steps
+        args.warmup = 3 if args.warmup is None else args.warmup
         run_reference(args, wl)
         return
-    if args.warmup < 3:
-        args.warmup = 3
+    args.steps = 1000 if args.steps is None else args.steps
+    args.warmup = max(3, 50 if args.warmup is None else args.warmup)
 
     import paper_2007_14062_b200 as bb
 
@@ -228,13 +249,15 @@ def main():
         torch.cuda.synchronize()
 
     L = bb.bigbird_build_layout(wl.N, wl.b, wl.w, wl.g, wl.r, wl.seed, wl.H, wl.mode)
-    pairs = counted_pairs(L, wl)
+    pairs = counted_pairs(L)
     flops_per_step = wl.B * pairs * 4.0 * wl.b * wl.b * wl.D
     tokens_per_step = wl.B * wl.N
 
     # Rotating input sets so that no step finds its inputs in L2 (4 sets x 201 MB for the base workload; L2 is 126 MB).
     q, k, v = synth.make_qkv(wl)
     kpm = synth.key_padding_mask(wl)
+    eff_pairs = effective_pairs(L, wl, kpm)
+    eff_flops_per_step = eff_pairs * 4.0 * wl.b * wl.b * wl.D
     n_sets = 4
     sets = []
     for i in range(n_sets):
@@ -343,12 +366,14 @@ def main():
             "metric": METRIC, "value": tflops, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
-            "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "N": wl.N, "D": wl.D, "block": wl.b, "window_blocks": wl.w,
-                       "global_blocks": wl.g, "random_blocks": wl.r, "mode": "ETC" if wl.mode else "ITC",
-                       "attended_block_pairs_per_step": wl.B * pairs, "counted_gflop_per_step": flops_per_step / 1e9,
-                       "l2": f"rotating {n_sets} input/output sets ({n_sets * 4 * q.numel() * 2 / 1e6:.0f} MB) larger than L2",
-                       "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
+            "config": dict(workload_config(wl, pairs),
+                           effective_block_pairs_per_step=eff_pairs, effective_gflop_per_step=eff_flops_per_step / 1e9,
+                           l2=f"rotating {n_sets} input/output sets ({n_sets * 4 * q.numel() * q.element_size() / 1e6:.0f} MB) larger than L2",
+                           parallelism=f"replicas x{world}" if world > 1 else "single GPU"),
             "tokens_per_s": world * tokens_per_step / (ms_per_step * 1e-3),
+            # the same time against the pairs that survive the key-padding mask (equal to `value` without padding)
+            "effective_tflops": tflops * eff_flops_per_step / flops_per_step,
+            "pct_of_measured_bf16_peak_effective": 100.0 * per_gpu * eff_flops_per_step / flops_per_step / peaks["bf16_tflops"],
             "pct_of_measured_bf16_peak": 100.0 * per_gpu / peaks["bf16_tflops"],
             "pct_of_nominal_bf16_peak": 100.0 * per_gpu / NOMINAL_BF16_TFLOPS,
             "e2e": {"value": e2e_tflops, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
