@@ -209,6 +209,79 @@ def run_reference(args, wl):
     }))
 
 
+def run_backward(args, wl):
+    """`--direction bwd`: the gradient kernels (CUDA cores, fp32 arithmetic) on the same workload, one GPU.  Their
+    FLOPs are counted like the forward pass's: five b x b x D products per attended block pair (the scores again,
+    dP, dV, dQ, dK) against the forward pass's two."""
+    import paper_2007_14062_b200 as bb
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    steps = 20 if args.steps is None else args.steps
+    warmup = max(3, 3 if args.warmup is None else args.warmup)
+    L = bb.bigbird_build_layout(wl.N, wl.b, wl.w, wl.g, wl.r, wl.seed, wl.H, wl.mode)
+    pairs = counted_pairs(L)
+    flops_per_step = wl.B * pairs * 10.0 * wl.b * wl.b * wl.D
+    q, k, v = synth.make_qkv(wl)
+    kpm = synth.key_padding_mask(wl)
+    gen = torch.Generator().manual_seed(wl.seed + 100)
+    dout = torch.randn(q.shape, generator=gen, dtype=torch.float32).to(q.dtype)
+    qd, kd, vd, dod = (t.to(dev) for t in (q, k, v, dout))
+    md = None if kpm is None else kpm.to(dev)
+    out, lse = torch.empty_like(qd), torch.empty(q.shape[:3], device=dev, dtype=torch.float32)
+    bb.bigbird_attn_fwd(qd, kd, vd, L, md, out, lse, wl.scale)
+    dq, dk, dv = (torch.empty_like(qd) for _ in range(3))
+    stream = torch.cuda.current_stream(dev)
+
+    def step():
+        bb.bigbird_attn_bwd(qd, kd, vd, out, lse, dod, L, md, dq, dk, dv, wl.scale, stream.cuda_stream)
+
+    for _ in range(warmup):
+        step()
+    launches = bb.bigbird_last_launch_count()
+    sampler = ClockSampler(0)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    sampler.start()
+    ev0.record(stream)
+    for _ in range(steps):
+        step()
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    sampler.stop()
+    ms_per_step = ev0.elapsed_time(ev1) / steps
+    tflops = flops_per_step / (ms_per_step * 1e-3) / 1e12
+    clocks = sampler.summary()
+    # fp32 FMA peak of the CUDA cores from unit counts and the clock: SMs x 128 lanes x 2 FLOP x max SM clock
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    alu_peak = sms * 128 * 2 * (clocks["sm_max_mhz"] or 1965) * 1e6 / 1e12
+    elt = q.element_size()
+    min_bytes = wl.B * wl.H * wl.N * (8 * wl.D * elt + 4)          # q, k, v, out, dout read, dq, dk, dv written, lse read
+    line = {"metric": "block-sparse attn bwd TFLOP/s (counted FLOPs)", "value": tflops, "unit": UNIT, "n_gpus": 1, "steps": steps,
+            "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic", "direction": "bwd",
+            "config": dict(workload_config(wl, pairs), counted_gflop_per_step_bwd=flops_per_step / 1e9,
+                           l2=f"one set of eight tensors ({8 * q.numel() * elt / 1e6:.0f} MB)"),
+            "gpu_launches": launches * steps, "clocks": clocks,
+            "roofline": {"bound": "alu", "achieved": tflops, "peak": alu_peak, "unit": "TFLOP/s", "frac": tflops / alu_peak,
+                         "traffic": None, "peak_source": "fp32 FMA lanes x clock (derived)", "kernel": "attn_bwd_dq_kernel + attn_bwd_dkv_kernel",
+                         "min_hbm_bytes_per_launch": min_bytes, "achieved_hbm_gbs_on_min_bytes": min_bytes / (ms_per_step * 1e-3) / 1e9}}
+    if not args.no_cpu_baseline:
+        from oracle import bigbird_oracle as O
+        gr = O.Graph(wl.N, wl.b, wl.w, wl.g, wl.r, wl.seed, wl.H, wl.mode)
+        t0 = time.perf_counter()
+        want = O.attention_bwd(q[:1].float().numpy(), k[:1].float().numpy(), v[:1].float().numpy(), dout[:1].float().numpy(), gr,
+                               None if kpm is None else kpm[:1].numpy(), wl.scale, slices=[(0, 0)])
+        t = time.perf_counter() - t0
+        got = [x[0, 0].float().cpu().numpy() for x in (dq, dk, dv)]
+        err = max(float(np.abs(g - w_).max()) for g, w_ in zip(got, want[(0, 0)]))
+        line["cpu_baseline"] = {"value": flops_per_step / (wl.B * wl.H) / t / 1e12, "unit": UNIT, "cores": len(os.sched_getaffinity(0)),
+                                "kind": "oracle", "sample": f"1 of {wl.B * wl.H} (batch, head) slices, fp64 gradients; {t:.2f} s",
+                                "max_abs_err_grads_vs_oracle": err}
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -218,6 +291,7 @@ def main():
     ap.add_argument("--workload", default="c2_base_itc_bf16", choices=synth.ORDER)
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--direction", default="fwd", choices=["fwd", "bwd"], help="bwd: time the gradient kernels instead (one GPU)")
     args = ap.parse_args()
     wl = synth.WORKLOADS[args.workload]
 
@@ -225,6 +299,10 @@ def main():
         args.steps = 12 if args.steps is None else args.steps
         args.warmup = 3 if args.warmup is None else args.warmup
         run_reference(args, wl)
+        return
+    if args.direction == "bwd":
+        if int(os.environ.get("RANK", "0")) == 0:
+            run_backward(args, wl)
         return
     args.steps = 1000 if args.steps is None else args.steps
     args.warmup = max(3, 50 if args.warmup is None else args.warmup)
