@@ -34,6 +34,21 @@ def test_layout_sweep_bit_exact():
         L.close()
 
 
+@pytest.mark.parametrize("cfg", [(84 * (3 + 49), 84, 3, 3, 0, 0, 12, 1),      # ETC base: block 84, 4116 tokens + 3 global blocks
+                                 (169 * (3 + 24), 169, 3, 3, 0, 0, 16, 1),    # QA large: block 169, 4056 tokens + 3 global blocks
+                                 (84 * 49, 84, 3, 2, 3, 5, 4, 0)])            # the same block size with random blocks, ITC
+def test_layout_of_the_papers_etc_block_sizes_bit_exact(cfg):
+    """Block sizes of the paper's ETC settings (App. E hyper-parameter tables): the graph is built in blocks, so only
+    N % b == 0 matters; the global token count is rounded up to whole blocks by the caller and the tail masked."""
+    L = bb.bigbird_build_layout(*cfg)
+    rp, ci = L.export()
+    orp, oci = _oracle_csr(*cfg)
+    assert np.array_equal(rp, orp) and np.array_equal(ci, oci)
+    cp, ri = L.export_transposed()
+    assert cp[-1] == rp[-1] and len(ri) == len(ci)
+    L.close()
+
+
 def test_library_random_blocks_match_hand_worked_vectors():
     """The library's own selection against the hand-worked vectors of tests/golden/random_blocks_seed0.txt
     (App. D item 1 under the generator spec of bigbird.h), independently of the oracle."""

@@ -105,6 +105,38 @@ def test_small_cases_every_element(wl, impl):
     _compare(wl, q, k, v, kpm, out, lse, slices=None)
 
 
+# The paper's own ETC settings have block sizes that are not powers of two and global token counts that are not whole
+# blocks (App. E hyper-parameter tables: ETC base, block 84, 230 global tokens, window 252 = 3 blocks; QA large, block
+# 169, 430 global tokens, window 507 = 3 blocks; no random blocks).  The CUDA-core path takes any block size; the
+# global tokens take the first g = 3 blocks and the unused tail of the third one is masked out as padding, which is the
+# same graph for the tokens that exist.
+PAPER_ETC = [
+    ("etc_base_b84", synth.Workload("etc_b84", "fp32", 1, 2, 84 * (3 + 9), 64, 84, 3, 3, 0, 1, seed=21), 230),
+    ("etc_base_b84_bf16", synth.Workload("etc_b84_bf16", "bf16", 2, 2, 84 * (3 + 7), 64, 84, 3, 3, 0, 1, seed=22), 230),
+    ("qa_large_b169", synth.Workload("qa_b169", "fp32", 1, 2, 169 * (3 + 5), 64, 169, 3, 3, 0, 1, seed=23), 430),
+]
+
+
+@pytest.mark.parametrize("name,wl,g_tokens", PAPER_ETC, ids=[c[0] for c in PAPER_ETC])
+def test_paper_etc_block_sizes_on_the_cuda_core_path(name, wl, g_tokens):
+    q, k, v = synth.make_qkv(wl)
+    kpm = torch.ones(wl.B, wl.N, dtype=torch.uint8)
+    kpm[:, g_tokens:wl.g * wl.b] = 0                           # the global slots beyond the paper's count
+    if wl.B > 1:
+        kpm[1, wl.N - 100:] = 0                                # and a shorter sequence
+    out, lse = _run(wl, q, k, v, kpm, "simt")
+    _compare(wl, q, k, v, kpm, out, lse, slices=None)
+    # the tensor-core entry point says so instead of computing something else
+    if wl.dtype == "bf16":
+        dev = torch.device("cuda:0")
+        L = bb.bigbird_build_layout(wl.N, wl.b, wl.w, wl.g, wl.r, wl.seed, wl.H, wl.mode)
+        qd = q.to(dev)
+        with pytest.raises(bb.BigBirdError) as ei:
+            bb.bigbird_attn_fwd(qd, qd, qd, L, None, torch.empty_like(qd), None, wl.scale)
+        assert ei.value.code == -2                              # BIGBIRD_EUNSUPPORTED
+        L.close()
+
+
 @pytest.mark.parametrize("impl", ["fwd", "simt"])
 def test_fully_padded_sequence_and_no_lse(impl):
     wl = _small("bf16", 2, 2, 8)
