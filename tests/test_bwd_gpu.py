@@ -26,6 +26,7 @@ CASES = [
     _case("bf16", 2, 2, 12, lengths="ragged:100:768"),
     _case("bf16", 1, 2, 9, mode=1, r=0),
     _case("fp32", 1, 2, 8, b=84, mode=1, g=3, r=0),             # the paper's ETC block size (App. E tables)
+    _case("fp32", 1, 2, 6, D=128),                              # the largest head dimension of the CUDA-core kernels
 ]
 
 

@@ -105,6 +105,16 @@ def test_small_cases_every_element(wl, impl):
     _compare(wl, q, k, v, kpm, out, lse, slices=None)
 
 
+# Head dimensions other than 64 exist on the CUDA-core path only (the tensor-core kernel is D = 64).
+@pytest.mark.parametrize("dtype,D", [("fp32", 128), ("bf16", 128), ("fp32", 32)])
+def test_other_head_dimensions_on_the_cuda_core_path(dtype, D):
+    wl = synth.Workload(f"headdim_{dtype}_{D}", dtype, 2, 2, 9 * 64, D, 64, 3, 2, 3, 0, seed=31, lengths="ragged:100:576")
+    q, k, v = synth.make_qkv(wl)
+    kpm = synth.key_padding_mask(wl)
+    out, lse = _run(wl, q, k, v, kpm, "simt")
+    _compare(wl, q, k, v, kpm, out, lse, slices=None)
+
+
 # The paper's own ETC settings have block sizes that are not powers of two and global token counts that are not whole
 # blocks (App. E hyper-parameter tables: ETC base, block 84, 230 global tokens, window 252 = 3 blocks; QA large, block
 # 169, 430 global tokens, window 507 = 3 blocks; no random blocks).  The CUDA-core path takes any block size; the
