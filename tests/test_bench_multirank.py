@@ -40,3 +40,32 @@ def test_single_process_and_aggregate_value():
     assert bench.max_over_ranks([1.5, 2.5], None, None) == [1.5, 2.5]
     # 4 replicas, 10 units each per step, slowest step 2 ms -> 20000 units/s
     assert bench.whole_job_value(10.0, 4, 2.0) == 20000.0
+
+
+def test_effective_pairs_count_what_survives_the_padding_mask():
+    """bench.py's effective FLOP count against the oracle's token-level mask: a (query block, key block) pair of the
+    layout counts if some valid query row of the block attends some valid key of the key block."""
+    sys.path.insert(0, ROOT)
+    import numpy as np
+    import bench
+    import paper_2007_14062_b200 as bb
+    from paper_2007_14062_b200 import synth
+    from oracle import bigbird_oracle as O
+    wl = synth.Workload("eff", "bf16", 3, 2, 10 * 64, 64, 64, 3, 2, 3, 0, seed=5, lengths="ragged:64:640")
+    L = bb.bigbird_build_layout(wl.N, wl.b, wl.w, wl.g, wl.r, wl.seed, wl.H, wl.mode)
+    kpm = synth.key_padding_mask(wl)
+    kpm[1, 130:] = 0                                            # a length that is not a multiple of the block size
+    kpm[1, :130] = 1
+    got = bench.effective_pairs(L, wl, kpm)
+    gr = O.Graph(wl.N, wl.b, wl.w, wl.g, wl.r, wl.seed, wl.H, wl.mode)
+    want = 0
+    nb = wl.N // wl.b
+    for h in range(wl.H):
+        A = O.build_mask(gr, h)                                 # [N, N] 0/1, token level
+        for bi in range(wl.B):
+            valid = kpm[bi].numpy() != 0
+            M = A.astype(bool) & valid[:, None] & valid[None, :]
+            want += int(M.reshape(nb, wl.b, nb, wl.b).any(axis=(1, 3)).sum())
+    assert got == want
+    assert bench.effective_pairs(L, wl, None) == wl.B * bench.counted_pairs(L)
+    L.close()
